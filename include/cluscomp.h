@@ -1,0 +1,187 @@
+/*
+ * cluscomp.h -- C ABI of the B200 (sm_100a) clustering library.
+ *
+ * The library computes the clustering step of ClusComp (Section 3.1,
+ * "ClusComp-: Clustering"): the sub-vectors of a weight matrix are clustered by
+ * Lloyd's k-means into a codebook C (n centroids of dimension g) and codes q
+ * (one index per sub-vector); Section 3.2 fixes the storage (FP16 codebook,
+ * unsigned 16-bit codes) and the appendix listing fixes the reshape / decode
+ * layout.
+ *
+ * Conventions for every call below
+ *  - Pointers are DEVICE pointers owned by the caller unless the name ends in
+ *    `_host`.  FP16 data is passed as uint16_t bit patterns (IEEE binary16).
+ *  - `stream` is a cudaStream_t passed as void* (NULL = the default stream).
+ *    Calls enqueue work on it and return without waiting; outputs are valid
+ *    after the stream has been synchronised.
+ *  - Arguments are validated on the host before anything is launched.  A call
+ *    that returns a status other than CC_OK has enqueued nothing and its
+ *    outputs are undefined.  The library never aborts and its kernels never
+ *    trap; problems found on the device (non-finite input) are recorded in a
+ *    status word that cc_poll_status() reads back.
+ *  - N = number of sub-vectors, g = sub-vector dimension (1..16),
+ *    K = number of centroids (1..65536, the paper keeps n <= 2^16 so that a
+ *    code fits 16 bits; codes are 0-based).  N < 2^31.
+ *  - The same inputs give bit-identical outputs on every call.
+ *  - Scratch memory is one caller-owned workspace (cc_workspace_bytes /
+ *    cc_set_workspace); the library itself allocates no device memory except
+ *    in cc_compress_host.
+ */
+#ifndef CLUSCOMP_H_
+#define CLUSCOMP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    CC_OK = 0,
+    CC_ERR_NULL = 1,           /* a required pointer is NULL                              */
+    CC_ERR_SHAPE = 2,          /* a size is <= 0 or too large                             */
+    CC_ERR_UNSUPPORTED_G = 3,  /* g outside 1..16                                         */
+    CC_ERR_K_RANGE = 4,        /* K outside 1..65536                                      */
+    CC_ERR_N_LT_K = 5,         /* initialisation needs K distinct sub-vectors             */
+    CC_ERR_ALIGN = 6,          /* X / C / W pointers must be 16-byte aligned              */
+    CC_ERR_WORKSPACE = 7,      /* no workspace set, or smaller than cc_workspace_bytes    */
+    CC_ERR_NONFINITE = 8,      /* Inf / NaN met in the input (reported by cc_poll_status) */
+    CC_ERR_DEVICE_TIMEOUT = 9, /* a bounded device-side wait ran out                      */
+    CC_ERR_CUDA = 10,          /* a CUDA runtime call failed                              */
+    CC_ERR_LAYOUT = 11         /* unknown layout / path constant                          */
+} cc_status;
+
+/* How sub-vectors are cut out of W (d_out x d_in, row-major, as a linear layer stores it). */
+#define CC_LAYOUT_PAPER_T 0 /* W' = W^T.view(-1, g): g consecutive out_features at a fixed
+                               in_feature; out_features zero-padded to a multiple of g
+                               (Section 3.1 footnote; "deficiency" in the appendix listing). */
+#define CC_LAYOUT_ROWS 1    /* W' = W.view(-1, g): g consecutive in_features of one row;
+                               in_features zero-padded to a multiple of g.                   */
+
+/* Which E-step kernel family cc_assign uses. */
+#define CC_PATH_AUTO 0   /* chosen per (g, K) from measurements                        */
+#define CC_PATH_FFMA 1   /* FP32 FMA pipes, register-tiled                             */
+#define CC_PATH_TENSOR 2 /* tcgen05 tensor cores with TMEM accumulators (g = 4, 8, 16) */
+
+typedef struct cc_ctx cc_ctx; /* opaque; one per device and per concurrent user */
+
+/* Context.  cc_create binds to `device` (cudaSetDevice is called inside every entry point).
+ * cc_destroy frees only host state; the workspace stays the caller's. */
+cc_status cc_create(cc_ctx** out, int device);
+cc_status cc_destroy(cc_ctx* ctx);
+const char* cc_status_string(cc_status s);
+
+/* Scratch memory needed by any call on a problem of this size, in bytes (0 on bad arguments).
+ * The workspace must stay valid and unshared while calls using it are in flight. */
+size_t cc_workspace_bytes(int64_t N, int g, int K);
+cc_status cc_set_workspace(cc_ctx* ctx, void* workspace, size_t bytes);
+
+/* CC_PATH_* override for cc_assign / cc_fit / cc_finalize (default CC_PATH_AUTO).
+ * Every path returns the same idx and counts. */
+cc_status cc_set_path(cc_ctx* ctx, int path);
+
+/* Number of kernels this context has launched so far (host counter). */
+int64_t cc_launch_count(const cc_ctx* ctx);
+
+/* Measurement aids (no counterpart in the paper).  With timing enabled every kernel launch is
+ * bracketed by a CUDA event pair on its own stream (at most 8192 launches between two reads).
+ * cc_profile_read waits for those events, adds up the device time and the number of launches
+ * of one kernel class, for all classes at once: total_ms_host / launches_host are host arrays
+ * of CC_KERNEL_CLASSES entries (either may be NULL), and the record is cleared. */
+#define CC_KERNEL_ASSIGN_MAIN 0   /* the N x K distance scan of the E-step              */
+#define CC_KERNEL_ASSIGN_PREP 1   /* staging of the codebook for the scan               */
+#define CC_KERNEL_RESOLVE 2       /* exact FP64 stage for near-ties                     */
+#define CC_KERNEL_OBJECTIVE 3     /* deterministic sum of the distances                 */
+#define CC_KERNEL_UPDATE_ACCUM 4  /* M-step: integer sums and counts                    */
+#define CC_KERNEL_UPDATE_FINISH 5 /* M-step: division, empty-cluster rule               */
+#define CC_KERNEL_RESHAPE 6
+#define CC_KERNEL_DECODE 7
+#define CC_KERNEL_OTHER 8
+#define CC_KERNEL_CLASSES 9
+cc_status cc_profile_enable(cc_ctx* ctx, int on);
+cc_status cc_profile_read(cc_ctx* ctx, double* total_ms_host, int64_t* launches_host);
+
+/* Runs a register-only FP32 FMA loop on every SM (the ceiling the FP32 E-step is measured
+ * against) and returns the achieved TFLOP/s (2 flops per FMA) for the scalar and the packed
+ * two-wide instruction form.  Synchronises `stream`.  Outputs are host doubles. */
+cc_status cc_measure_fp32_peak(cc_ctx* ctx, double* tflops_scalar_host, double* tflops_packed_host,
+                               void* stream);
+
+/* Host helpers.  Number of sub-vectors after padding: the appendix listing's
+ * num_codes = in_features * (out_features + deficiency) / g (PAPER_T), or the same rule along
+ * in_features (ROWS); -1 on bad arguments.  Average bits per parameter, Eq. 1 of Section 3.2:
+ * (16 * codes + 16 * g * K) / (d_in * d_out), codes counted after padding. */
+int64_t cc_num_subvectors(int64_t d_out, int64_t d_in, int g, int layout);
+double cc_bits_per_param(int64_t d_out, int64_t d_in, int g, int K);
+
+/* Section 3.1 (footnote) / appendix listing: cut W into sub-vectors.
+ * W: d_out x d_in FP16 row-major.  X (out): N x g FP16 row-major, N = cc_num_subvectors(...);
+ * padded elements are +0.  W and X must not overlap. */
+cc_status cc_reshape_subvectors(cc_ctx* ctx, const uint16_t* W, int64_t d_out, int64_t d_in, int g,
+                                int layout, uint16_t* X, void* stream);
+
+/* Initial codebook.  The paper leaves this to its library's defaults; the rule here: K distinct
+ * positions from a partial Fisher-Yates shuffle of 0..N-1 driven by splitmix64(seed)
+ * (for i < K: j = i + next() mod (N - i); swap a[i], a[j]; position i is a[i]);
+ * C[k] = X[position k] widened to FP32.  cc_init_positions writes the K positions to host memory
+ * (no device work).  C (out): K x g FP32.  Needs 1 <= K <= N. */
+cc_status cc_init_positions(int64_t N, int K, uint64_t seed, int64_t* positions_host);
+cc_status cc_init_codebook(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, int K, uint64_t seed,
+                           float* C, void* stream);
+
+/* E-step of Section 3.1: idx[i] = the centroid minimising ||x_i - c_j||^2 (lowest j on exact
+ * ties), dist[i] = that squared distance (FP32), *objective = sum_i dist[i] (the Section 3.1
+ * objective for this assignment, a plain sum).  X: N x g FP16; C: K x g FP32.
+ * idx (out): N x uint16.  dist (out, may be NULL): N x FP32.  objective (out, device, may be
+ * NULL): one double.  n_resolved (out, device, may be NULL): one int64 = how many points had
+ * their two best FP32 scores closer than the rounding bound and were decided in FP64.
+ * N = 0 is allowed (objective 0). */
+cc_status cc_assign(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const float* C, int K,
+                    uint16_t* idx, float* dist, double* objective, int64_t* n_resolved, void* stream);
+
+/* M-step of Section 3.1: counts[j] = |{i : idx[i] = j}| (exact), C[j] = mean of those x_i
+ * (exact integer sum, one rounding to FP32); a cluster with no member keeps its centroid
+ * bit for bit (the paper does not say; this library's rule).  C: in = previous, out = new.
+ * counts (out): K x int32.  idx values must be < K. */
+cc_status cc_update(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const uint16_t* idx, int K,
+                    float* C, int32_t* counts, void* stream);
+
+/* Lloyd loop of Section 3.1: iters x (E-step, M-step), no early stop (the paper runs a fixed
+ * 20).  C: in = initial, out = after the last M-step.  idx / dist / counts (out): those of the
+ * last iteration.  objective_trace (out, device, may be NULL): iters doubles, entry t = the
+ * objective at the t-th E-step.  N >= 1, iters >= 0. */
+cc_status cc_fit(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, int K, int iters, float* C,
+                 uint16_t* idx, float* dist, int32_t* counts, double* objective_trace, void* stream);
+
+/* Section 3.1 (codes = nearest centroid of the final codebook) and Section 3.2 (FP16 storage):
+ * C16 = round-to-nearest-even FP16 of C; idx / dist / objective = E-step against C16, so the
+ * stored pair (C16, idx) is consistent and ||W - decode||^2 equals *objective (no padding). */
+cc_status cc_finalize(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const float* C, int K,
+                      uint16_t* C16, uint16_t* idx, float* dist, double* objective, void* stream);
+
+/* Reconstruction, Section 3.1 / appendix listing (codebook[code].view(in_features, -1) with
+ * the padded columns dropped): W_hat (out): d_out x d_in FP16 row-major, the layout of W.
+ * idx: cc_num_subvectors(...) codes, each < K. */
+cc_status cc_decode(cc_ctx* ctx, const uint16_t* C16, int K, int g, const uint16_t* idx,
+                    int64_t d_out, int64_t d_in, int layout, uint16_t* W_hat, void* stream);
+
+/* Waits for `stream`, reads the device status word and clears it.  Returns CC_OK,
+ * CC_ERR_NONFINITE, CC_ERR_DEVICE_TIMEOUT or CC_ERR_CUDA. */
+cc_status cc_poll_status(cc_ctx* ctx, void* stream);
+
+/* Whole path on HOST buffers (Sections 3.1-3.2 end to end): copies W to the device, reshapes,
+ * initialises, runs `iters` Lloyd iterations, finalises, and copies the FP16 codebook, the
+ * codes and the final objective back; optionally also decodes into W_hat_host (may be NULL).
+ * Allocates and frees its own device buffers and workspace and synchronises before returning.
+ * All pointers are host pointers (pinned memory makes the copies asynchronous).
+ * objective_trace_host (may be NULL): iters + 1 doubles, the last being the final objective. */
+cc_status cc_compress_host(cc_ctx* ctx, const uint16_t* W_host, int64_t d_out, int64_t d_in, int g,
+                           int K, int iters, uint64_t seed, int layout, uint16_t* C16_host,
+                           uint16_t* idx_host, double* objective_trace_host, uint16_t* W_hat_host,
+                           void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CLUSCOMP_H_ */

@@ -1,0 +1,375 @@
+// C ABI of the library: host-side validation, workspace carving, the Lloyd loop.
+// Every step of the path runs in the kernels of the other translation units; nothing here
+// computes on the host except the seeded choice of the K initial positions.
+#include <new>
+#include <unordered_map>
+#include <vector>
+
+#include "cc_common.cuh"
+
+WsLayout cc_ws_layout(int64_t N, int g, int K) {
+    WsLayout L;
+    size_t off = 0;
+    auto take = [&](size_t bytes) { size_t o = off; off += cc_align_up(bytes ? bytes : 1, 256); return o; };
+    const size_t Kpad = cc_align_up((size_t)K, CC_KPAD);
+    L.status = take(256);
+    L.cprep = take(Kpad / 2 * (size_t)(g + 1) * 16);
+    L.flagged = take((size_t)N * 4);
+    L.partials = take((size_t)CC_OBJ_BLOCKS * 8);
+    L.sum_lo = take((size_t)K * g * 8);
+    L.sum_hi = take((size_t)K * g * 8);
+    L.tmp_c = take((size_t)K * g * 4);
+    L.positions = take((size_t)K * 8);
+    L.dist_tmp = take((size_t)N * 4);
+    // tensor-core staging: split codebook operand (Kpad x 64 floats at most) + squared norms
+    L.tensor = take(Kpad * (size_t)(64 + 1) * 4);
+    L.total = off;
+    return L;
+}
+
+namespace {
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+cc_status check_common(const cc_ctx* ctx, int64_t N, int g, int K, bool need_ws) {
+    if (!ctx) return CC_ERR_NULL;
+    if (g < 1 || g > 16) return CC_ERR_UNSUPPORTED_G;
+    if (K < 1 || K > 65536) return CC_ERR_K_RANGE;
+    if (N < 0 || N >= (int64_t)1 << 31) return CC_ERR_SHAPE;
+    if (need_ws) {
+        if (!ctx->ws) return CC_ERR_WORKSPACE;
+        if (ctx->ws_bytes < cc_ws_layout(N, g, K).total) return CC_ERR_WORKSPACE;
+    }
+    return CC_OK;
+}
+
+inline cc_status from_cuda(cudaError_t e) { return e == cudaSuccess ? CC_OK : CC_ERR_CUDA; }
+
+inline uint64_t splitmix64(uint64_t& s) {
+    uint64_t z = (s += 0x9E3779B97F4A7C15ull);
+    z = (z ^ (z >> 30)) * 0xBF58476D1CE4E5B9ull;
+    z = (z ^ (z >> 27)) * 0x94D049BB133111EBull;
+    return z ^ (z >> 31);
+}
+
+// Only the K touched entries of the shuffled array are kept (a map from position to content).
+void partial_shuffle(int64_t N, int K, uint64_t seed, int64_t* pos) {
+    std::unordered_map<int64_t, int64_t> moved;
+    moved.reserve((size_t)K * 2);
+    uint64_t s = seed;
+    for (int64_t i = 0; i < K; ++i) {
+        const int64_t j = i + (int64_t)(splitmix64(s) % (uint64_t)(N - i));
+        auto itj = moved.find(j);
+        const int64_t vj = (itj == moved.end()) ? j : itj->second;
+        auto iti = moved.find(i);
+        const int64_t vi = (iti == moved.end()) ? i : iti->second;
+        moved[j] = vi;
+        moved[i] = vj;
+        pos[i] = vj;
+    }
+}
+
+bool use_tensor_path(const cc_ctx* ctx, int g, int K) {
+    if (ctx->path == CC_PATH_FFMA) return false;
+    if (!cc_tensor_path_supported(g, K)) return false;
+    return true;   // AUTO and TENSOR: the tensor-core kernels win wherever they apply
+}
+
+cudaError_t assign_any(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64_t N, int g, const float* C, int K,
+                       uint16_t* idx, float* dist, double* objective, int64_t* n_resolved, cudaStream_t st) {
+    if (!dist) dist = reinterpret_cast<float*>(static_cast<char*>(ctx->ws) + L.dist_tmp);
+    if (use_tensor_path(ctx, g, K))
+        return cc_launch_assign_tensor(ctx, L, X, N, g, C, K, idx, dist, objective, n_resolved, st);
+    return cc_launch_assign_ffma(ctx, L, X, N, g, C, K, idx, dist, objective, n_resolved, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+const char* cc_status_string(cc_status s) {
+    switch (s) {
+        case CC_OK: return "ok";
+        case CC_ERR_NULL: return "null pointer";
+        case CC_ERR_SHAPE: return "bad size";
+        case CC_ERR_UNSUPPORTED_G: return "g outside 1..16";
+        case CC_ERR_K_RANGE: return "K outside 1..65536";
+        case CC_ERR_N_LT_K: return "fewer sub-vectors than centroids";
+        case CC_ERR_ALIGN: return "pointer not 16-byte aligned";
+        case CC_ERR_WORKSPACE: return "workspace missing or too small";
+        case CC_ERR_NONFINITE: return "non-finite input";
+        case CC_ERR_DEVICE_TIMEOUT: return "device-side wait ran out";
+        case CC_ERR_CUDA: return "CUDA runtime error";
+        case CC_ERR_LAYOUT: return "unknown layout or path";
+    }
+    return "unknown status";
+}
+
+cc_status cc_create(cc_ctx** out, int device) {
+    if (!out) return CC_ERR_NULL;
+    *out = nullptr;
+    int n = 0;
+    if (cudaGetDeviceCount(&n) != cudaSuccess || device < 0 || device >= n) return CC_ERR_CUDA;
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return CC_ERR_CUDA;
+    cc_ctx* c = new (std::nothrow) cc_ctx();
+    if (!c) return CC_ERR_CUDA;
+    c->device = device;
+    c->sm_count = prop.multiProcessorCount;
+    c->path = CC_PATH_AUTO;
+    c->ws = nullptr;
+    c->ws_bytes = 0;
+    c->launches = 0;
+    c->pos_host = nullptr;
+    c->pos_cap = 0;
+    c->prof_on = 0;
+    c->prof_used = c->prof_made = 0;
+    c->prof = nullptr;
+    *out = c;
+    return CC_OK;
+}
+
+cc_status cc_destroy(cc_ctx* ctx) {
+    if (!ctx) return CC_ERR_NULL;
+    delete[] ctx->pos_host;
+    if (ctx->prof) {
+        cudaSetDevice(ctx->device);
+        for (int i = 0; i < ctx->prof_made; ++i) { cudaEventDestroy(ctx->prof[i].a); cudaEventDestroy(ctx->prof[i].b); }
+        delete[] ctx->prof;
+    }
+    delete ctx;
+    return CC_OK;
+}
+
+size_t cc_workspace_bytes(int64_t N, int g, int K) {
+    if (g < 1 || g > 16 || K < 1 || K > 65536 || N < 0 || N >= (int64_t)1 << 31) return 0;
+    return cc_ws_layout(N, g, K).total;
+}
+
+cc_status cc_set_workspace(cc_ctx* ctx, void* workspace, size_t bytes) {
+    if (!ctx) return CC_ERR_NULL;
+    if (workspace && (!aligned16(workspace) || bytes < 256)) return CC_ERR_ALIGN;
+    ctx->ws = workspace;
+    ctx->ws_bytes = workspace ? bytes : 0;
+    if (workspace) {
+        if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+        if (cudaMemset(workspace, 0, 256) != cudaSuccess) return CC_ERR_CUDA;   // status words
+    }
+    return CC_OK;
+}
+
+cc_status cc_set_path(cc_ctx* ctx, int path) {
+    if (!ctx) return CC_ERR_NULL;
+    if (path != CC_PATH_AUTO && path != CC_PATH_FFMA && path != CC_PATH_TENSOR) return CC_ERR_LAYOUT;
+    ctx->path = path;
+    return CC_OK;
+}
+
+int64_t cc_launch_count(const cc_ctx* ctx) { return ctx ? ctx->launches : -1; }
+
+int64_t cc_num_subvectors(int64_t d_out, int64_t d_in, int g, int layout) {
+    if (d_out < 1 || d_in < 1 || g < 1) return -1;
+    if (layout == CC_LAYOUT_PAPER_T) return d_in * ((d_out + g - 1) / g);
+    if (layout == CC_LAYOUT_ROWS) return d_out * ((d_in + g - 1) / g);
+    return -1;
+}
+
+double cc_bits_per_param(int64_t d_out, int64_t d_in, int g, int K) {
+    const int64_t codes = cc_num_subvectors(d_out, d_in, g, CC_LAYOUT_PAPER_T);
+    if (codes < 0 || K < 1) return -1.0;
+    return (16.0 * (double)codes + 16.0 * (double)g * (double)K) / ((double)d_in * (double)d_out);
+}
+
+cc_status cc_reshape_subvectors(cc_ctx* ctx, const uint16_t* W, int64_t d_out, int64_t d_in, int g, int layout,
+                                uint16_t* X, void* stream) {
+    if (!ctx || !W || !X) return CC_ERR_NULL;
+    if (g < 1 || g > 16) return CC_ERR_UNSUPPORTED_G;
+    if (layout != CC_LAYOUT_PAPER_T && layout != CC_LAYOUT_ROWS) return CC_ERR_LAYOUT;
+    const int64_t N = cc_num_subvectors(d_out, d_in, g, layout);
+    if (N < 1 || N >= (int64_t)1 << 31) return CC_ERR_SHAPE;
+    if (!aligned16(W) || !aligned16(X)) return CC_ERR_ALIGN;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    return from_cuda(cc_launch_reshape(ctx, W, d_out, d_in, g, layout, X, (cudaStream_t)stream));
+}
+
+cc_status cc_init_positions(int64_t N, int K, uint64_t seed, int64_t* positions_host) {
+    if (!positions_host) return CC_ERR_NULL;
+    if (K < 1 || K > 65536) return CC_ERR_K_RANGE;
+    if (N < 1 || N >= (int64_t)1 << 31) return CC_ERR_SHAPE;
+    if (N < K) return CC_ERR_N_LT_K;
+    partial_shuffle(N, K, seed, positions_host);
+    return CC_OK;
+}
+
+cc_status cc_init_codebook(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, int K, uint64_t seed, float* C,
+                           void* stream) {
+    if (!ctx || !X || !C) return CC_ERR_NULL;
+    cc_status s = check_common(ctx, N, g, K, true);
+    if (s != CC_OK) return s;
+    if (N < 1) return CC_ERR_SHAPE;
+    if (N < K) return CC_ERR_N_LT_K;
+    if (!aligned16(X) || !aligned16(C)) return CC_ERR_ALIGN;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    if (ctx->pos_cap < K) {
+        delete[] ctx->pos_host;
+        ctx->pos_host = new (std::nothrow) int64_t[K];
+        ctx->pos_cap = ctx->pos_host ? K : 0;
+        if (!ctx->pos_host) return CC_ERR_CUDA;
+    }
+    partial_shuffle(N, K, seed, ctx->pos_host);
+    const WsLayout L = cc_ws_layout(N, g, K);
+    int64_t* pos_dev = reinterpret_cast<int64_t*>(static_cast<char*>(ctx->ws) + L.positions);
+    cudaStream_t st = (cudaStream_t)stream;
+    // pageable source: the copy is staged before the call returns, so pos_host may be reused
+    if (cudaMemcpyAsync(pos_dev, ctx->pos_host, sizeof(int64_t) * (size_t)K, cudaMemcpyHostToDevice, st) !=
+        cudaSuccess)
+        return CC_ERR_CUDA;
+    return from_cuda(cc_launch_gather_init(ctx, X, g, K, pos_dev, C, st));
+}
+
+cc_status cc_assign(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const float* C, int K, uint16_t* idx,
+                    float* dist, double* objective, int64_t* n_resolved, void* stream) {
+    if (!ctx || !C || (N > 0 && (!X || !idx))) return CC_ERR_NULL;
+    cc_status s = check_common(ctx, N, g, K, true);
+    if (s != CC_OK) return s;
+    if (!aligned16(X) || !aligned16(C)) return CC_ERR_ALIGN;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    const WsLayout L = cc_ws_layout(N, g, K);
+    return from_cuda(assign_any(ctx, L, X, N, g, C, K, idx, dist, objective, n_resolved, (cudaStream_t)stream));
+}
+
+cc_status cc_update(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const uint16_t* idx, int K, float* C,
+                    int32_t* counts, void* stream) {
+    if (!ctx || !C || !counts || (N > 0 && (!X || !idx))) return CC_ERR_NULL;
+    cc_status s = check_common(ctx, N, g, K, true);
+    if (s != CC_OK) return s;
+    if (!aligned16(X) || !aligned16(C)) return CC_ERR_ALIGN;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    const WsLayout L = cc_ws_layout(N, g, K);
+    return from_cuda(cc_launch_update(ctx, L, X, N, g, idx, K, C, counts, (cudaStream_t)stream));
+}
+
+cc_status cc_fit(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, int K, int iters, float* C, uint16_t* idx,
+                 float* dist, int32_t* counts, double* objective_trace, void* stream) {
+    if (!ctx || !X || !C || !idx || !counts) return CC_ERR_NULL;
+    cc_status s = check_common(ctx, N, g, K, true);
+    if (s != CC_OK) return s;
+    if (N < 1 || iters < 0) return CC_ERR_SHAPE;
+    if (!aligned16(X) || !aligned16(C)) return CC_ERR_ALIGN;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    const WsLayout L = cc_ws_layout(N, g, K);
+    cudaStream_t st = (cudaStream_t)stream;
+    for (int it = 0; it < iters; ++it) {
+        cudaError_t e = assign_any(ctx, L, X, N, g, C, K, idx, dist, objective_trace ? objective_trace + it : nullptr,
+                                   nullptr, st);
+        if (e != cudaSuccess) return CC_ERR_CUDA;
+        e = cc_launch_update(ctx, L, X, N, g, idx, K, C, counts, st);
+        if (e != cudaSuccess) return CC_ERR_CUDA;
+    }
+    return CC_OK;
+}
+
+cc_status cc_finalize(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const float* C, int K, uint16_t* C16,
+                      uint16_t* idx, float* dist, double* objective, void* stream) {
+    if (!ctx || !X || !C || !C16 || !idx) return CC_ERR_NULL;
+    cc_status s = check_common(ctx, N, g, K, true);
+    if (s != CC_OK) return s;
+    if (N < 1) return CC_ERR_SHAPE;
+    if (!aligned16(X) || !aligned16(C) || !aligned16(C16)) return CC_ERR_ALIGN;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    const WsLayout L = cc_ws_layout(N, g, K);
+    cudaStream_t st = (cudaStream_t)stream;
+    float* widened = reinterpret_cast<float*>(static_cast<char*>(ctx->ws) + L.tmp_c);
+    cudaError_t e = cc_launch_to_half(ctx, C, (int64_t)K * g, C16, widened, st);
+    if (e != cudaSuccess) return CC_ERR_CUDA;
+    return from_cuda(assign_any(ctx, L, X, N, g, widened, K, idx, dist, objective, nullptr, st));
+}
+
+cc_status cc_decode(cc_ctx* ctx, const uint16_t* C16, int K, int g, const uint16_t* idx, int64_t d_out,
+                    int64_t d_in, int layout, uint16_t* W_hat, void* stream) {
+    if (!ctx || !C16 || !idx || !W_hat) return CC_ERR_NULL;
+    if (g < 1 || g > 16) return CC_ERR_UNSUPPORTED_G;
+    if (K < 1 || K > 65536) return CC_ERR_K_RANGE;
+    if (layout != CC_LAYOUT_PAPER_T && layout != CC_LAYOUT_ROWS) return CC_ERR_LAYOUT;
+    const int64_t N = cc_num_subvectors(d_out, d_in, g, layout);
+    if (N < 1 || N >= (int64_t)1 << 31) return CC_ERR_SHAPE;
+    if (!aligned16(C16) || !aligned16(W_hat)) return CC_ERR_ALIGN;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    return from_cuda(cc_launch_decode(ctx, C16, K, g, idx, d_out, d_in, layout, W_hat, (cudaStream_t)stream));
+}
+
+cc_status cc_poll_status(cc_ctx* ctx, void* stream) {
+    if (!ctx) return CC_ERR_NULL;
+    if (!ctx->ws) return CC_ERR_WORKSPACE;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned word = 0;
+    if (cudaMemcpyAsync(&word, ctx->ws, sizeof(word), cudaMemcpyDeviceToHost, st) != cudaSuccess) return CC_ERR_CUDA;
+    if (cudaMemsetAsync(ctx->ws, 0, sizeof(word), st) != cudaSuccess) return CC_ERR_CUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return CC_ERR_CUDA;
+    if (word & CC_DEV_TIMEOUT) return CC_ERR_DEVICE_TIMEOUT;
+    if (word & CC_DEV_NONFINITE) return CC_ERR_NONFINITE;
+    return CC_OK;
+}
+
+cc_status cc_compress_host(cc_ctx* ctx, const uint16_t* W_host, int64_t d_out, int64_t d_in, int g, int K, int iters,
+                           uint64_t seed, int layout, uint16_t* C16_host, uint16_t* idx_host,
+                           double* objective_trace_host, uint16_t* W_hat_host, void* stream) {
+    if (!ctx || !W_host || !C16_host || !idx_host) return CC_ERR_NULL;
+    if (g < 1 || g > 16) return CC_ERR_UNSUPPORTED_G;
+    if (K < 1 || K > 65536) return CC_ERR_K_RANGE;
+    if (layout != CC_LAYOUT_PAPER_T && layout != CC_LAYOUT_ROWS) return CC_ERR_LAYOUT;
+    if (iters < 0) return CC_ERR_SHAPE;
+    const int64_t N = cc_num_subvectors(d_out, d_in, g, layout);
+    if (N < 1 || N >= (int64_t)1 << 31) return CC_ERR_SHAPE;
+    if (N < K) return CC_ERR_N_LT_K;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    const size_t w_bytes = (size_t)d_out * d_in * 2, x_bytes = (size_t)N * g * 2;
+    const size_t ws_bytes = cc_ws_layout(N, g, K).total;
+    // one allocation, carved: W | X | C | C16 | idx | dist | counts | trace | workspace
+    size_t off = 0;
+    auto take = [&](size_t b) { size_t o = off; off += cc_align_up(b, 256); return o; };
+    const size_t oW = take(w_bytes), oX = take(x_bytes), oC = take((size_t)K * g * 4), oC16 = take((size_t)K * g * 2),
+                 oIdx = take((size_t)N * 2), oDist = take((size_t)N * 4), oCnt = take((size_t)K * 4),
+                 oTr = take((size_t)(iters + 1) * 8), oWs = take(ws_bytes);
+    char* base = nullptr;
+    if (cudaMalloc(&base, off) != cudaSuccess) return CC_ERR_CUDA;
+    void* saved_ws = ctx->ws;
+    const size_t saved_bytes = ctx->ws_bytes;
+    cc_status s = cc_set_workspace(ctx, base + oWs, ws_bytes);
+    uint16_t* W = (uint16_t*)(base + oW);
+    uint16_t* X = (uint16_t*)(base + oX);
+    float* C = (float*)(base + oC);
+    uint16_t* C16 = (uint16_t*)(base + oC16);
+    uint16_t* idx = (uint16_t*)(base + oIdx);
+    float* dist = (float*)(base + oDist);
+    int32_t* counts = (int32_t*)(base + oCnt);
+    double* trace = (double*)(base + oTr);
+    if (s == CC_OK && cudaMemcpyAsync(W, W_host, w_bytes, cudaMemcpyHostToDevice, st) != cudaSuccess) s = CC_ERR_CUDA;
+    if (s == CC_OK) s = cc_reshape_subvectors(ctx, W, d_out, d_in, g, layout, X, st);
+    if (s == CC_OK) s = cc_init_codebook(ctx, X, N, g, K, seed, C, st);
+    if (s == CC_OK) s = cc_fit(ctx, X, N, g, K, iters, C, idx, dist, counts, trace, st);
+    if (s == CC_OK) s = cc_finalize(ctx, X, N, g, C, K, C16, idx, dist, trace + iters, st);
+    if (s == CC_OK && W_hat_host) {
+        s = cc_decode(ctx, C16, K, g, idx, d_out, d_in, layout, W, st);   // W is no longer needed
+        if (s == CC_OK && cudaMemcpyAsync(W_hat_host, W, w_bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            s = CC_ERR_CUDA;
+    }
+    if (s == CC_OK && cudaMemcpyAsync(C16_host, C16, (size_t)K * g * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        s = CC_ERR_CUDA;
+    if (s == CC_OK && cudaMemcpyAsync(idx_host, idx, (size_t)N * 2, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        s = CC_ERR_CUDA;
+    if (s == CC_OK && objective_trace_host &&
+        cudaMemcpyAsync(objective_trace_host, trace, (size_t)(iters + 1) * 8, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+        s = CC_ERR_CUDA;
+    if (s == CC_OK) s = cc_poll_status(ctx, st);
+    else cudaStreamSynchronize(st);
+    ctx->ws = saved_ws;
+    ctx->ws_bytes = saved_bytes;
+    cudaFree(base);
+    return s;
+}
+
+}  // extern "C"

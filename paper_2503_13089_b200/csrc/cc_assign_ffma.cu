@@ -1,0 +1,461 @@
+// E-step of Section 3.1 on the FP32 FMA pipes, plus the exact second stage and the
+// objective sum that both E-step paths share.
+//
+// Fast stage.  For point x and centroid c the comparison score is
+//     s = ||c||^2 - 2 x.c        (||x||^2 is the same for every centroid and dropped)
+// computed as one FMA chain  s = fma(x_{g-1}, m_{g-1}, ... fma(x_0, m_0, csq))  with m = -2c and
+// csq = ||c||^2 staged once per call.  Each thread keeps P points in registers (as f32x2 pairs of
+// two points) and walks the staged codebook through shared memory; every shared-memory value is
+// read by the whole warp at once (a broadcast).  Only the running MINIMUM of the scores is kept
+// in the inner loop (one 3-input min per two scores); the minimum is tracked per chunk of CHUNK
+// centroids, together with the best and second-best chunk minima, and the winning chunk is
+// rescanned once per point at the end to recover the index and the runner-up inside it.
+//
+// Exactness.  |s_computed - s| <= gamma_{g+1} (2||c||^2 + ||x||^2) with gamma_n ~ n 2^-24.  For any
+// centroid at least as close as the fast winner b, ||c||^2 <= 2||x||^2 + 2 d_b^2, so if the gap
+// between the two smallest computed scores exceeds 2 gamma (5||x||^2 + 4 d_b^2) the fast winner is
+// the true nearest centroid.  Otherwise the point is appended to a list and decided again by the
+// exact stage (FP64, direct form, lowest index on ties).  The N x K matrix is never stored.
+#include <float.h>
+
+#include "cc_common.cuh"
+
+namespace {
+
+typedef unsigned long long ull;
+
+__device__ __forceinline__ ull pack2(float lo, float hi) {
+    ull r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(ull v, float& lo, float& hi) {
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+// Two FP32 FMAs in one instruction (sm_100 packed form); each lane rounds like fma.rn.f32.
+__device__ __forceinline__ ull fma2(ull a, ull b, ull c) {
+    ull d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+__device__ __forceinline__ float min3(float a, float b, float c) {
+    float d;
+    asm("min.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
+__device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
+    unsigned s = (unsigned)__cvta_generic_to_shared(smem);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(s), "l"(gmem));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+
+constexpr float kBig = 3.0e38f;   // score of the padding centroids; above any real score
+constexpr int kThreads = 256;
+
+template <int G> struct FfmaCfg {
+    static constexpr int P = (G <= 8) ? 8 : 4;                       // points per thread
+    static constexpr int TILE = (G <= 4) ? 512 : (G <= 8) ? 256 : 128;  // centroids per smem tile
+    static constexpr int CHUNK = 32;                                  // centroids per tracked minimum
+    static constexpr int ROW4 = G + 1;                                // float4 per centroid pair
+};
+
+// Load one point (G halves) as floats; rows beyond N read as zeros.
+template <int G>
+__device__ __forceinline__ void load_point(const uint16_t* __restrict__ X, int64_t i, int64_t N, float* x,
+                                           bool& nonfinite) {
+    if (i >= N) {
+#pragma unroll
+        for (int t = 0; t < G; ++t) x[t] = 0.f;
+        return;
+    }
+    const uint16_t* row = X + i * G;
+    uint16_t h[G];
+    if constexpr (G % 8 == 0) {
+#pragma unroll
+        for (int v = 0; v < G / 8; ++v) {
+            uint4 u = __ldg(reinterpret_cast<const uint4*>(row) + v);
+            unsigned w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) { h[v * 8 + 2 * k] = w[k] & 0xffffu; h[v * 8 + 2 * k + 1] = w[k] >> 16; }
+        }
+    } else if constexpr (G % 4 == 0) {
+#pragma unroll
+        for (int v = 0; v < G / 4; ++v) {
+            uint2 u = __ldg(reinterpret_cast<const uint2*>(row) + v);
+            h[v * 4] = u.x & 0xffffu; h[v * 4 + 1] = u.x >> 16; h[v * 4 + 2] = u.y & 0xffffu; h[v * 4 + 3] = u.y >> 16;
+        }
+    } else if constexpr (G % 2 == 0) {
+#pragma unroll
+        for (int v = 0; v < G / 2; ++v) {
+            unsigned u = __ldg(reinterpret_cast<const unsigned*>(row) + v);
+            h[v * 2] = u & 0xffffu; h[v * 2 + 1] = u >> 16;
+        }
+    } else {
+#pragma unroll
+        for (int t = 0; t < G; ++t) h[t] = __ldg(row + t);
+    }
+#pragma unroll
+    for (int t = 0; t < G; ++t) {
+        if ((h[t] & 0x7c00u) == 0x7c00u) nonfinite = true;
+        x[t] = __half2float(__ushort_as_half(h[t]));
+    }
+}
+
+// Staged codebook: for each pair of centroids (2q, 2q+1), G float4 {m_{2q,t}, m_{2q,t}, m_{2q+1,t},
+// m_{2q+1,t}} followed by {csq_{2q}, csq_{2q}, csq_{2q+1}, csq_{2q+1}}; m = -2c.  Each value appears
+// twice so that one 128-bit shared load yields two ready f32x2 operands (one per centroid, the same
+// value for both points of a pair).  Centroids K..Kpad-1 are padding that can never win.
+template <int G>
+__global__ void prep_ffma_kernel(const float* __restrict__ C, int K, int Kpad, float4* __restrict__ prep,
+                                 unsigned* __restrict__ status) {
+    int q = blockIdx.x * blockDim.x + threadIdx.x;
+    if (q == 0) {  // reset the flagged-point counter of this E-step
+        *reinterpret_cast<ull*>(status + 2) = 0ull;
+    }
+    if (q >= Kpad / 2) return;
+    float m[2][G], csq[2];
+#pragma unroll
+    for (int h = 0; h < 2; ++h) {
+        int j = 2 * q + h;
+        if (j < K) {
+            double s = 0.0;
+#pragma unroll
+            for (int t = 0; t < G; ++t) {
+                float c = C[(int64_t)j * G + t];
+                m[h][t] = -2.0f * c;
+                s += (double)c * (double)c;
+            }
+            csq[h] = (float)s;
+        } else {
+#pragma unroll
+            for (int t = 0; t < G; ++t) m[h][t] = 0.f;
+            csq[h] = kBig;
+        }
+    }
+    float4* out = prep + (int64_t)q * (G + 1);
+#pragma unroll
+    for (int t = 0; t < G; ++t) out[t] = make_float4(m[0][t], m[0][t], m[1][t], m[1][t]);
+    out[G] = make_float4(csq[0], csq[0], csq[1], csq[1]);
+}
+
+template <int G>
+__global__ void __launch_bounds__(kThreads, (G <= 4) ? 2 : 1)
+assign_ffma_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restrict__ C, int K, int Kpad,
+                   const float4* __restrict__ prep, uint16_t* __restrict__ idx, float* __restrict__ dist,
+                   unsigned* __restrict__ status, unsigned* __restrict__ flagged) {
+    using Cfg = FfmaCfg<G>;
+    constexpr int P = Cfg::P, TILE = Cfg::TILE, CHUNK = Cfg::CHUNK, ROW4 = Cfg::ROW4;
+    constexpr int TILE4 = TILE / 2 * ROW4;   // float4 per tile
+    static_assert(P * kThreads * 2 * 4 <= 2 * TILE4 * 16, "stash must fit in the tile buffers");
+    __shared__ float4 tiles[2][TILE4];
+
+    const int tid = threadIdx.x;
+    const int64_t base = (int64_t)blockIdx.x * (kThreads * P);
+
+    // ---- points of this thread, as pairs (point 2pp, point 2pp+1) per dimension
+    ull xp[P / 2][G];
+    bool nonfinite = false;
+#pragma unroll
+    for (int pp = 0; pp < P / 2; ++pp) {
+        float xa[G], xb[G];
+        load_point<G>(X, base + (int64_t)(2 * pp) * kThreads + tid, N, xa, nonfinite);
+        load_point<G>(X, base + (int64_t)(2 * pp + 1) * kThreads + tid, N, xb, nonfinite);
+#pragma unroll
+        for (int t = 0; t < G; ++t) xp[pp][t] = pack2(xa[t], xb[t]);
+    }
+    if (nonfinite) atomicOr(status, CC_DEV_NONFINITE);
+
+    float b1[P], b2[P];
+    int bc[P];
+#pragma unroll
+    for (int p = 0; p < P; ++p) { b1[p] = INFINITY; b2[p] = INFINITY; bc[p] = 0; }
+
+    const int n_tiles = Kpad / TILE;
+    // prefetch tile 0
+    for (int e = tid; e < TILE4; e += kThreads) cp_async16(&tiles[0][e], prep + e);
+    cp_async_commit();
+
+    for (int tile = 0; tile < n_tiles; ++tile) {
+        cp_async_wait_all();
+        __syncthreads();   // tile `tile` has landed for everyone; buffer (tile+1)&1 is free again
+        if (tile + 1 < n_tiles) {
+            const float4* src = prep + (int64_t)(tile + 1) * TILE4;
+            float4* dst = tiles[(tile + 1) & 1];
+            for (int e = tid; e < TILE4; e += kThreads) cp_async16(dst + e, src + e);
+            cp_async_commit();
+        }
+        const float4* tbuf = tiles[tile & 1];
+#pragma unroll 1
+        for (int c = 0; c < TILE / CHUNK; ++c) {
+            float m[P];
+#pragma unroll
+            for (int p = 0; p < P; ++p) m[p] = INFINITY;
+            const float4* cp = tbuf + c * (CHUNK / 2) * ROW4;
+#pragma unroll 2
+            for (int q = 0; q < CHUNK / 2; ++q) {
+                const float4* row = cp + q * ROW4;
+                float4 cs = row[G];
+                ull accA[P / 2], accB[P / 2];
+                const ull csA = pack2(cs.x, cs.y), csB = pack2(cs.z, cs.w);
+#pragma unroll
+                for (int t = 0; t < G; ++t) {
+                    float4 mv = row[t];
+                    const ull mA = pack2(mv.x, mv.y), mB = pack2(mv.z, mv.w);
+#pragma unroll
+                    for (int pp = 0; pp < P / 2; ++pp) {
+                        accA[pp] = fma2(xp[pp][t], mA, t == 0 ? csA : accA[pp]);
+                        accB[pp] = fma2(xp[pp][t], mB, t == 0 ? csB : accB[pp]);
+                    }
+                }
+#pragma unroll
+                for (int pp = 0; pp < P / 2; ++pp) {
+                    float a0, a1, c0, c1;
+                    unpack2(accA[pp], a0, a1);
+                    unpack2(accB[pp], c0, c1);
+                    m[2 * pp] = min3(m[2 * pp], a0, c0);
+                    m[2 * pp + 1] = min3(m[2 * pp + 1], a1, c1);
+                }
+            }
+            const int chunk_id = tile * (TILE / CHUNK) + c;
+#pragma unroll
+            for (int p = 0; p < P; ++p) {
+                const bool better = m[p] < b1[p];
+                b2[p] = better ? b1[p] : fminf(b2[p], m[p]);
+                bc[p] = better ? chunk_id : bc[p];
+                b1[p] = better ? m[p] : b1[p];
+            }
+        }
+    }
+    __syncthreads();   // everyone is done with the tile buffers: reuse them as a stash
+
+    float* stash = reinterpret_cast<float*>(&tiles[0][0]);
+#pragma unroll
+    for (int p = 0; p < P; ++p) {
+        stash[(0 * P + p) * kThreads + tid] = b2[p];
+        stash[(1 * P + p) * kThreads + tid] = __int_as_float(bc[p]);
+    }
+    // (each thread reads back only what it wrote: no barrier needed)
+
+    constexpr double kErr = 2.0 * (G + 2) * 5.9604644775390625e-8;   // 2 * gamma_{g+1}, with margin
+#pragma unroll 1
+    for (int p = 0; p < P; ++p) {
+        const int64_t i = base + (int64_t)p * kThreads + tid;
+        if (i >= N) continue;
+        const float second_other = stash[(0 * P + p) * kThreads + tid];
+        const int chunk = __float_as_int(stash[(1 * P + p) * kThreads + tid]);
+        float x[G];
+        bool nf = false;
+        load_point<G>(X, i, N, x, nf);
+        // rescan the winning chunk: same FMA chain, ascending j, strict '<' keeps the lowest index
+        float s1 = INFINITY, s2 = INFINITY;
+        int j1 = chunk * CHUNK;
+        const float4* cp = prep + (int64_t)chunk * (CHUNK / 2) * ROW4;
+#pragma unroll 2
+        for (int q = 0; q < CHUNK / 2; ++q) {
+            const float4* row = cp + q * ROW4;
+            float4 cs = __ldg(row + G);
+            float sa = cs.x, sb = cs.z;
+#pragma unroll
+            for (int t = 0; t < G; ++t) {
+                float4 mv = __ldg(row + t);
+                sa = fmaf(x[t], mv.x, sa);
+                sb = fmaf(x[t], mv.z, sb);
+            }
+            const int j = chunk * CHUNK + 2 * q;
+            if (sa < s1) { s2 = s1; s1 = sa; j1 = j; } else if (sa < s2) s2 = sa;
+            if (sb < s1) { s2 = s1; s1 = sb; j1 = j + 1; } else if (sb < s2) s2 = sb;
+        }
+        if (j1 >= K) j1 = K - 1;   // only reachable with non-finite input
+        s2 = fminf(s2, second_other);
+        // squared distance to the winner, direct form in FP64 (no contraction)
+        double A = 0.0, D = 0.0;
+#pragma unroll
+        for (int t = 0; t < G; ++t) {
+            const double xd = (double)x[t];
+            const double df = __dsub_rn(xd, (double)__ldg(C + (int64_t)j1 * G + t));
+            D = __dadd_rn(D, __dmul_rn(df, df));
+            A = __dadd_rn(A, __dmul_rn(xd, xd));
+        }
+        idx[i] = (uint16_t)j1;
+        dist[i] = (float)D;
+        const double gap = (double)s2 - (double)s1;
+        if (!(gap > kErr * (5.0 * A + 4.0 * D))) {
+            const ull slot = atomicAdd(reinterpret_cast<ull*>(status + 2), 1ull);
+            flagged[slot] = (unsigned)i;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Exact stage: one thread per flagged point scans every centroid.  A cheap FP32 direct-form
+// distance (relative error <= (g+2) 2^-24, no cancellation) screens the candidates; those within
+// 2^-18 of the best FP64 distance so far are recomputed in FP64 (sub, mul, add, in dimension
+// order, no FMA contraction) and the pair (distance, index) is minimised lexicographically.
+template <int G>
+__global__ void __launch_bounds__(64)
+resolve_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restrict__ C, int K,
+               const unsigned* __restrict__ status, const unsigned* __restrict__ flagged,
+               uint16_t* __restrict__ idx, float* __restrict__ dist) {
+    ull F = *reinterpret_cast<const ull*>(status + 2);
+    if (F > (ull)N) F = (ull)N;
+    for (ull f = (ull)blockIdx.x * blockDim.x + threadIdx.x; f < F; f += (ull)gridDim.x * blockDim.x) {
+        const int64_t i = flagged[f];
+        float x[G];
+        bool nf = false;
+        load_point<G>(X, i, N, x, nf);
+        int jb = idx[i];
+        double Db = 0.0;
+#pragma unroll
+        for (int t = 0; t < G; ++t) {
+            const double df = __dsub_rn((double)x[t], (double)__ldg(C + (int64_t)jb * G + t));
+            Db = __dadd_rn(Db, __dmul_rn(df, df));
+        }
+        float bound = __double2float_ru(Db * (1.0 + 3.814697265625e-6));
+#pragma unroll 4
+        for (int j = 0; j < K; ++j) {
+            float c[G];
+#pragma unroll
+            for (int t = 0; t < G; ++t) c[t] = __ldg(C + (int64_t)j * G + t);
+            float dh = 0.f;
+#pragma unroll
+            for (int t = 0; t < G; ++t) { const float df = x[t] - c[t]; dh = fmaf(df, df, dh); }
+            if (dh <= bound) {
+                double d = 0.0;
+#pragma unroll
+                for (int t = 0; t < G; ++t) {
+                    const double df = __dsub_rn((double)x[t], (double)c[t]);
+                    d = __dadd_rn(d, __dmul_rn(df, df));
+                }
+                if (d < Db || (d == Db && j < jb)) {
+                    Db = d; jb = j;
+                    bound = __double2float_ru(Db * (1.0 + 3.814697265625e-6));
+                }
+            }
+        }
+        idx[i] = (uint16_t)jb;
+        dist[i] = (float)Db;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Objective: sum of dist in FP64 with a fixed summation tree (same bits on every run).
+__device__ __forceinline__ double block_sum(double v, double* sh) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_down_sync(0xffffffffu, v, o);
+    const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
+    if (l == 0) sh[w] = v;
+    __syncthreads();
+    double r = 0.0;
+    if (w == 0) {
+        r = (l < (blockDim.x >> 5)) ? sh[l] : 0.0;
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) r += __shfl_down_sync(0xffffffffu, r, o);
+    }
+    return r;   // valid in thread 0
+}
+
+__global__ void __launch_bounds__(256)
+objective_partial_kernel(const float* __restrict__ dist, int64_t N, double* __restrict__ partials) {
+    __shared__ double sh[8];
+    const int64_t per = (N + gridDim.x - 1) / gridDim.x;
+    const int64_t lo = (int64_t)blockIdx.x * per;
+    const int64_t hi = (lo + per < N) ? lo + per : N;
+    double acc = 0.0;
+    for (int64_t i = lo + threadIdx.x; i < hi; i += blockDim.x) acc += (double)dist[i];
+    const double r = block_sum(acc, sh);
+    if (threadIdx.x == 0) partials[blockIdx.x] = r;
+}
+
+__global__ void __launch_bounds__(256)
+objective_final_kernel(const double* __restrict__ partials, int n, const unsigned* __restrict__ status,
+                       double* __restrict__ objective, int64_t* __restrict__ n_resolved) {
+    __shared__ double sh[8];
+    double acc = 0.0;
+    for (int i = threadIdx.x; i < n; i += blockDim.x) acc += partials[i];
+    const double r = block_sum(acc, sh);
+    if (threadIdx.x == 0) {
+        if (objective) *objective = r;
+        if (n_resolved) *n_resolved = (int64_t)*reinterpret_cast<const ull*>(status + 2);
+    }
+}
+
+template <int G>
+cudaError_t launch_ffma(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64_t N, const float* C, int K,
+                        uint16_t* idx, float* dist, cudaStream_t st) {
+    char* ws = static_cast<char*>(ctx->ws);
+    unsigned* status = reinterpret_cast<unsigned*>(ws + L.status);
+    float4* prep = reinterpret_cast<float4*>(ws + L.cprep);
+    unsigned* flagged = reinterpret_cast<unsigned*>(ws + L.flagged);
+    const int Kpad = (int)cc_align_up((size_t)K, CC_KPAD);
+    {
+        ProfScope ps(ctx, CC_K_ASSIGN_PREP, st);
+        prep_ffma_kernel<G><<<(Kpad / 2 + 127) / 128, 128, 0, st>>>(C, K, Kpad, prep, status);
+    }
+    if (N > 0) {
+        const int64_t per_block = (int64_t)kThreads * FfmaCfg<G>::P;
+        const int64_t blocks = (N + per_block - 1) / per_block;
+        ProfScope ps(ctx, CC_K_ASSIGN_MAIN, st);
+        assign_ffma_kernel<G><<<(unsigned)blocks, kThreads, 0, st>>>(X, N, C, K, Kpad, prep, idx, dist, status,
+                                                                     flagged);
+    }
+    return cudaGetLastError();
+}
+
+template <int G>
+cudaError_t launch_tail(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64_t N, const float* C, int K,
+                        uint16_t* idx, float* dist, double* objective, int64_t* n_resolved, cudaStream_t st) {
+    char* ws = static_cast<char*>(ctx->ws);
+    unsigned* status = reinterpret_cast<unsigned*>(ws + L.status);
+    unsigned* flagged = reinterpret_cast<unsigned*>(ws + L.flagged);
+    double* partials = reinterpret_cast<double*>(ws + L.partials);
+    if (N > 0) {
+        ProfScope ps(ctx, CC_K_RESOLVE, st);
+        resolve_kernel<G><<<ctx->sm_count * 8, 64, 0, st>>>(X, N, C, K, status, flagged, idx, dist);
+    }
+    if (objective || n_resolved) {
+        int blocks = (int)((N + 4095) / 4096);
+        if (blocks > CC_OBJ_BLOCKS) blocks = CC_OBJ_BLOCKS;
+        if (blocks > 0) {
+            ProfScope ps(ctx, CC_K_OBJECTIVE, st);
+            objective_partial_kernel<<<blocks, 256, 0, st>>>(dist, N, partials);
+        }
+        ProfScope ps(ctx, CC_K_OBJECTIVE, st);
+        objective_final_kernel<<<1, 256, 0, st>>>(partials, blocks, status, objective, n_resolved);
+    }
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+#define CC_DISPATCH_G(g, CALL)                                                                      \
+    switch (g) {                                                                                    \
+        case 1: CALL(1); break;   case 2: CALL(2); break;   case 3: CALL(3); break;                 \
+        case 4: CALL(4); break;   case 5: CALL(5); break;   case 6: CALL(6); break;                 \
+        case 7: CALL(7); break;   case 8: CALL(8); break;   case 9: CALL(9); break;                 \
+        case 10: CALL(10); break; case 11: CALL(11); break; case 12: CALL(12); break;               \
+        case 13: CALL(13); break; case 14: CALL(14); break; case 15: CALL(15); break;               \
+        case 16: CALL(16); break;                                                                   \
+        default: return cudaErrorInvalidValue;                                                      \
+    }
+
+cudaError_t cc_launch_assign_tail(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64_t N, int g,
+                                  const float* C, int K, uint16_t* idx, float* dist, double* objective,
+                                  int64_t* n_resolved, cudaStream_t st) {
+    cudaError_t e = cudaSuccess;
+#define CALL(G) e = launch_tail<G>(ctx, L, X, N, C, K, idx, dist, objective, n_resolved, st)
+    CC_DISPATCH_G(g, CALL)
+#undef CALL
+    return e;
+}
+
+cudaError_t cc_launch_assign_ffma(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64_t N, int g,
+                                  const float* C, int K, uint16_t* idx, float* dist, double* objective,
+                                  int64_t* n_resolved, cudaStream_t st) {
+    cudaError_t e = cudaSuccess;
+#define CALL(G) e = launch_ffma<G>(ctx, L, X, N, C, K, idx, dist, st)
+    CC_DISPATCH_G(g, CALL)
+#undef CALL
+    if (e != cudaSuccess) return e;
+    return cc_launch_assign_tail(ctx, L, X, N, g, C, K, idx, dist, objective, n_resolved, st);
+}

@@ -1,0 +1,99 @@
+// Shared host-side declarations of the library's translation units.
+#pragma once
+
+#include <cuda_fp16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "cluscomp.h"
+
+// Bits of the device status word (workspace, word 0).
+#define CC_DEV_NONFINITE 1u
+#define CC_DEV_TIMEOUT 2u
+
+// Kernel classes for the optional per-kernel event timing (cc_profile_*).
+enum { CC_K_ASSIGN_MAIN = 0, CC_K_ASSIGN_PREP = 1, CC_K_RESOLVE = 2, CC_K_OBJECTIVE = 3, CC_K_UPDATE_ACCUM = 4,
+       CC_K_UPDATE_FINISH = 5, CC_K_RESHAPE = 6, CC_K_DECODE = 7, CC_K_OTHER = 8, CC_K_COUNT = 9 };
+constexpr int CC_PROF_CAP = 8192;
+
+struct cc_prof_slot { cudaEvent_t a, b; int kind; };
+
+struct cc_ctx {
+    int device;
+    int sm_count;
+    int path;             // CC_PATH_*
+    void* ws;             // caller-owned workspace
+    size_t ws_bytes;
+    int64_t launches;     // kernels launched so far
+    int64_t* pos_host;    // staging for cc_init_codebook (K positions)
+    int pos_cap;
+    int prof_on;          // record an event pair around every kernel launch
+    int prof_used, prof_made;
+    cc_prof_slot* prof;   // CC_PROF_CAP slots, events created on first use
+};
+
+// Brackets one kernel launch with events on its stream when timing is enabled, and counts it.
+struct ProfScope {
+    cc_ctx* c; cudaStream_t st; cc_prof_slot* slot;
+    ProfScope(cc_ctx* ctx, int kind, cudaStream_t s) : c(ctx), st(s), slot(nullptr) {
+        c->launches++;
+        if (!c->prof_on || !c->prof || c->prof_used >= CC_PROF_CAP) return;
+        cc_prof_slot* sl = c->prof + c->prof_used;
+        if (c->prof_used >= c->prof_made) {
+            if (cudaEventCreate(&sl->a) != cudaSuccess || cudaEventCreate(&sl->b) != cudaSuccess) return;
+            c->prof_made = c->prof_used + 1;
+        }
+        sl->kind = kind;
+        cudaEventRecord(sl->a, st);
+        slot = sl;
+        c->prof_used++;
+    }
+    ~ProfScope() { if (slot) cudaEventRecord(slot->b, st); }
+};
+
+// Carving of the workspace for a problem (N, g, K).  All offsets 256-byte aligned.
+struct WsLayout {
+    size_t status;     // 64 x u32: [0] status bits, [2..3] flagged counter (u64)
+    size_t cprep;      // staged codebook for the FFMA E-step
+    size_t flagged;    // u32 list of points sent to the exact stage
+    size_t partials;   // doubles: per-block objective partial sums
+    size_t sum_lo;     // int64 K x g: sums of |x| < 8 in units of 2^-24
+    size_t sum_hi;     // int64 K x g: sums of |x| >= 8 in units of 2^-7
+    size_t tmp_c;      // float K x g: widened FP16 codebook (finalize)
+    size_t positions;  // int64 K: initial positions
+    size_t dist_tmp;   // float N: distances when the caller passes dist == NULL
+    size_t tensor;     // staging of the tensor-core E-step
+    size_t total;
+};
+
+constexpr int CC_KPAD = 1024;          // staged codebook is padded to a multiple of this
+constexpr int CC_OBJ_BLOCKS = 1024;    // partial sums of the objective reduction
+
+WsLayout cc_ws_layout(int64_t N, int g, int K);
+
+static inline size_t cc_align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+// Launchers (each returns cudaGetLastError() of its launches and bumps ctx->launches).
+cudaError_t cc_launch_reshape(cc_ctx*, const uint16_t* W, int64_t d_out, int64_t d_in, int g, int layout,
+                              uint16_t* X, cudaStream_t);
+cudaError_t cc_launch_decode(cc_ctx*, const uint16_t* C16, int K, int g, const uint16_t* idx, int64_t d_out,
+                             int64_t d_in, int layout, uint16_t* W_hat, cudaStream_t);
+cudaError_t cc_launch_gather_init(cc_ctx*, const uint16_t* X, int g, int K, const int64_t* pos_dev, float* C,
+                                  cudaStream_t);
+cudaError_t cc_launch_to_half(cc_ctx*, const float* C, int64_t n, uint16_t* C16, float* C_widened, cudaStream_t);
+
+cudaError_t cc_launch_assign_ffma(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const float* C,
+                                  int K, uint16_t* idx, float* dist, double* objective, int64_t* n_resolved,
+                                  cudaStream_t);
+bool cc_tensor_path_supported(int g, int K);
+cudaError_t cc_launch_assign_tensor(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const float* C,
+                                    int K, uint16_t* idx, float* dist, double* objective, int64_t* n_resolved,
+                                    cudaStream_t);
+// Second stage shared by both E-step paths: exact FP64 decision for the flagged points, then
+// the deterministic objective sum.
+cudaError_t cc_launch_assign_tail(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const float* C,
+                                  int K, uint16_t* idx, float* dist, double* objective, int64_t* n_resolved,
+                                  cudaStream_t);
+
+cudaError_t cc_launch_update(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const uint16_t* idx,
+                             int K, float* C, int32_t* counts, cudaStream_t);

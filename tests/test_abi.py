@@ -1,0 +1,66 @@
+"""Host-side checks of the C ABI that need no GPU: the library loads, exports every declared
+symbol, and its host helpers agree with the paper's printed values and with the oracle."""
+import os
+import re
+
+import numpy as np
+import pytest
+
+import oracle
+from paper_2503_13089_b200 import binding as cc
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "cluscomp.h")).read()
+    header = re.sub(r"/\*.*?\*/", "", header, flags=re.S)
+    declared = set(re.findall(r"\b(cc_[a-z0-9_]+)\s*\(", header))
+    assert len(declared) >= 20
+    lib = cc.load()
+    for name in sorted(declared):
+        assert hasattr(lib, name), name
+    assert declared == set(cc.SIGNATURES), declared ^ set(cc.SIGNATURES)
+
+
+def test_host_helpers_follow_listing_and_eq1():
+    for (o, i, g) in [(4096, 4096, 4), (4096, 4096, 6), (4096, 4096, 9), (10, 7, 4), (11008, 4096, 5)]:
+        for layout in (0, 1):
+            assert cc.cc_num_subvectors(o, i, g, layout) == oracle.num_subvectors(o, i, g, layout)
+        assert cc.cc_bits_per_param(o, i, g, 65500) == oracle.bits_per_param(o, i, g, 65500)
+    assert round(cc.cc_bits_per_param(4096, 4096, 4, 65500), 2) == 4.25      # printed in the paper's table
+    assert round(cc.cc_bits_per_param(4096, 4096, 6, 65500), 2) == 3.04
+    assert round(cc.cc_bits_per_param(4096, 4096, 9, 65500), 2) == 2.34
+    assert cc.cc_num_subvectors(0, 4, 4, 0) == -1 and cc.cc_num_subvectors(4, 4, 4, 9) == -1
+
+
+def test_init_positions_match_oracle_and_reject_bad_sizes():
+    for N, K, seed in [(1000003, 5, 1234567), (5000, 700, 42), (257, 257, 9), (58720256, 65536, 2004)]:
+        assert np.array_equal(cc.cc_init_positions(N, K, seed), oracle.init_positions(N, K, seed))
+    with pytest.raises(cc.CCError) as e:
+        cc.cc_init_positions(10, 11, 0)
+    assert e.value.status == 5
+    with pytest.raises(cc.CCError) as e:
+        cc.cc_init_positions(10, 0, 0)
+    assert e.value.status == 4
+    with pytest.raises(cc.CCError) as e:
+        cc.cc_init_positions(1 << 31, 4, 0)
+    assert e.value.status == 2
+
+
+def test_workspace_size_and_status_strings():
+    assert cc.cc_workspace_bytes(1000, 4, 16) > 0
+    assert cc.cc_workspace_bytes(1000, 17, 16) == 0 and cc.cc_workspace_bytes(1000, 4, 65537) == 0
+    assert cc.cc_workspace_bytes(-1, 4, 16) == 0
+    big = cc.cc_workspace_bytes(58720256, 4, 65536)
+    assert 2 * 58720256 * 4 <= big < 2 * 58720256 * 4 + (64 << 20)
+    assert cc.cc_status_string(0) == "ok" and "aligned" in cc.cc_status_string(6)
+
+
+def test_no_gpu_fails_loudly():
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("a GPU is present")
+    with pytest.raises(cc.CCError) as e:
+        cc.Context(0)
+    assert e.value.status == 10

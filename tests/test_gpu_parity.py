@@ -1,0 +1,337 @@
+"""GPU parity: the CUDA library against the CPU oracle, element by element, through the C ABI.
+
+Bars: indices / counts bit-exact (a differing index is tolerated only where the oracle's two
+distances differ by < 1e-6 relative, and is counted); centroids within 1e-4 relative max error;
+objective within 1e-5 relative.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2503_13089_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _cc():
+    from paper_2503_13089_b200 import binding
+    return binding
+
+
+def _u():
+    from tests import gpu_util
+    return gpu_util
+
+
+# ------------------------------------------------------------------ reshape / decode / init
+
+@pytest.mark.parametrize("layout", [0, 1])
+@pytest.mark.parametrize("d_out,d_in,g", [(8, 8, 4), (10, 7, 4), (130, 67, 4), (129, 200, 6), (64, 64, 16),
+                                          (100, 33, 9), (257, 300, 5), (1, 1, 1)])
+def test_reshape_and_decode_match_oracle(d_out, d_in, g, layout):
+    cc, u = _cc(), _u()
+    rng = np.random.default_rng(d_out + d_in + g)
+    W = rng.standard_normal((d_out, d_in)).astype(np.float16)
+    N = cc.cc_num_subvectors(d_out, d_in, g, layout)
+    assert N == oracle.num_subvectors(d_out, d_in, g, layout)
+    Wd = u.half_dev(W)
+    X = torch.full((N, g), 7.0, dtype=torch.float16, device="cuda")
+    cc.cc_reshape_subvectors(u.ctx(), Wd, d_out, d_in, g, layout, X)
+    Xo = oracle.reshape_subvectors(W, g, layout)
+    assert np.array_equal(u.u16_np(X.view(torch.uint16)).reshape(N, g), Xo.view(np.uint16))
+    K = 37
+    C16 = rng.standard_normal((K, g)).astype(np.float16)
+    idx = rng.integers(0, K, N).astype(np.uint16)
+    What = torch.zeros((d_out, d_in), dtype=torch.float16, device="cuda")
+    cc.cc_decode(u.ctx(), u.half_dev(C16), K, g, u.dev(idx.view(np.int16)).view(torch.uint16), d_out, d_in,
+                 layout, What)
+    want = oracle.decode(C16, idx.astype(np.int32), d_out, d_in, layout)
+    assert np.array_equal(u.u16_np(What.view(torch.uint16)).reshape(d_out, d_in), want.view(np.uint16))
+
+
+@pytest.mark.parametrize("N,g,K,seed", [(5000, 4, 700, 42), (257, 3, 257, 9), (100000, 8, 4096, 1)])
+def test_init_codebook_matches_oracle(N, g, K, seed):
+    cc, u = _cc(), _u()
+    X = wl.make_points(N, g, seed)
+    assert np.array_equal(cc.cc_init_positions(N, K, seed), oracle.init_positions(N, K, seed))
+    u.ctx().ensure_workspace(N, g, K)
+    C = torch.empty((K, g), dtype=torch.float32, device="cuda")
+    cc.cc_init_codebook(u.ctx(), u.half_dev(X), N, g, K, seed, C)
+    assert np.array_equal(C.cpu().numpy(), oracle.init_codebook(X, K, seed))
+
+
+# ------------------------------------------------------------------ E-step
+
+ASSIGN_CASES = [
+    # N, g, K   (tile = 2048 points x 128..512 centroids: several tiles and ragged tails)
+    (1, 4, 1), (31, 4, 2), (2049, 4, 33), (5000, 4, 255), (5000, 4, 257), (70001, 4, 1000),
+    (20000, 4, 4096), (3000, 4, 5000), (9000, 8, 300), (4097, 8, 2049), (6000, 16, 129),
+    (2500, 16, 1500), (3001, 1, 17), (3001, 2, 64), (3001, 3, 100), (3001, 5, 600), (3001, 6, 90),
+    (3001, 7, 1025), (3001, 9, 513), (1500, 12, 77), (1500, 13, 300), (1500, 15, 64),
+]
+
+
+@pytest.mark.parametrize("N,g,K", ASSIGN_CASES)
+def test_assign_matches_oracle(N, g, K):
+    u = _u()
+    X = wl.make_points(N, g, 1000 + N + g)
+    C = wl.make_codebook(K, g, 2000 + K + g)
+    idx, dist, obj, nres = u.gpu_assign(X, C)
+    tol, o_idx, d1 = u.check_assign_against_oracle(X, C, idx, dist)
+    assert tol <= max(1, N // 1000)
+    assert obj == pytest.approx(float(np.sum(dist.astype(np.float64))), rel=1e-12)
+    assert obj == pytest.approx(d1.sum(), rel=1e-6)
+    assert 0 <= nres <= N
+
+
+def test_assign_exact_ties_and_duplicates_take_lowest_index():
+    u = _u()
+    g, K, N = 4, 600, 4000
+    X = wl.make_points(N, g, 5)
+    C = wl.make_codebook(K, g, 6)
+    C[300:400] = C[100:200]                       # duplicated centroids
+    C[450] = C[3]
+    X[:K] = C.astype(np.float16)                  # points sitting (almost) on centroids
+    C[:64] = X[:64].astype(np.float32)            # ... and exactly on them
+    idx, dist, obj, nres = u.gpu_assign(X, C)
+    o_idx, d1, d2 = oracle.assign(X, C)
+    assert np.array_equal(idx, o_idx)             # exact ties included: no tolerance here
+    assert not np.any((idx >= 300) & (idx < 400)) and not np.any(idx == 450)
+    assert np.all(dist[:64] == 0)
+    assert nres >= 100
+
+
+def test_assign_lattice_points_with_many_exact_ties():
+    u = _u()
+    rng = np.random.default_rng(0)
+    X = (rng.integers(-3, 4, (6000, 4)) * 0.25).astype(np.float16)      # exactly representable grid
+    C = (rng.integers(-3, 4, (300, 4)) * 0.25 + 0.125).astype(np.float32)
+    idx, dist, obj, nres = u.gpu_assign(X, C)
+    o_idx, d1, _ = oracle.assign(X, C)
+    assert np.array_equal(idx, o_idx) and np.array_equal(dist, d1.astype(np.float32))
+
+
+def test_assign_empty_input_and_null_dist():
+    cc, u = _cc(), _u()
+    C = wl.make_codebook(10, 4, 1)
+    idx, dist, obj, nres = u.gpu_assign(np.zeros((0, 4), np.float16), C)
+    assert len(idx) == 0 and obj == 0.0 and nres == 0
+    X = wl.make_points(3000, 4, 2)
+    a = u.gpu_assign(X, C, want_dist=False)
+    b = u.gpu_assign(X, C)
+    assert np.array_equal(a[0], b[0]) and a[2] == b[2]
+
+
+def test_assign_metamorphic_scaling_and_determinism():
+    u = _u()
+    X = wl.make_points(30000, 4, 11)
+    C = wl.make_codebook(777, 4, 12)
+    a = u.gpu_assign(X, C)
+    b = u.gpu_assign(X, C)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1]) and a[2] == b[2] and a[3] == b[3]
+    Xs = (X.astype(np.float32) * 4).astype(np.float16)
+    s = u.gpu_assign(Xs, C * 4)
+    assert np.array_equal(s[0], a[0]) and np.array_equal(s[1], a[1] * 16)
+
+
+def test_assign_reports_nonfinite_input():
+    cc, u = _cc(), _u()
+    X = wl.make_points(5000, 4, 13)
+    X[1234, 2] = np.inf
+    with pytest.raises(cc.CCError) as e:
+        u.gpu_assign(X, wl.make_codebook(50, 4, 14))
+    assert e.value.status == 8
+    u.gpu_assign(wl.make_points(100, 4, 1), wl.make_codebook(5, 4, 1))   # status was cleared
+
+
+# ------------------------------------------------------------------ M-step
+
+@pytest.mark.parametrize("N,g,K", [(1, 4, 3), (5000, 4, 64), (70001, 4, 1000), (9000, 8, 5000), (6000, 16, 129),
+                                   (3001, 5, 17), (3001, 9, 200), (4000, 1, 7)])
+def test_update_matches_oracle_bit_for_bit(N, g, K):
+    u = _u()
+    X = wl.make_points(N, g, 3000 + N)
+    rng = np.random.default_rng(N)
+    idx = rng.integers(0, max(1, K - 2), N).astype(np.int32)      # the last clusters stay empty
+    C_prev = wl.make_codebook(K, g, 4000 + K)
+    C_or, counts_or = oracle.update(X, idx, C_prev)
+    C_gpu, counts_gpu = u.gpu_update(X, idx, C_prev)
+    assert np.array_equal(counts_gpu.astype(np.int64), counts_or)
+    assert u.centroid_rel_err(C_gpu, C_or, X) <= u.REL_CENTROID
+    assert np.array_equal(C_gpu.view(np.uint32), C_or.view(np.uint32))     # exact integer sums: same bits
+    assert np.array_equal(C_gpu[counts_or == 0].view(np.uint32), C_prev[counts_or == 0].view(np.uint32))
+
+
+def test_update_large_and_tiny_values_and_point_order():
+    u = _u()
+    rng = np.random.default_rng(3)
+    X = wl.make_points(20000, 4, 77)
+    X[::7] = (rng.standard_normal((len(X[::7]), 4)) * 300).astype(np.float16)       # |x| >= 8 accumulator
+    X[::11] = (rng.standard_normal((len(X[::11]), 4)) * 1e-6).astype(np.float16)    # subnormals
+    idx = rng.integers(0, 50, len(X)).astype(np.int32)
+    C_prev = np.zeros((50, 4), np.float32)
+    C_or, counts_or = oracle.update(X, idx, C_prev)
+    C_gpu, counts_gpu = u.gpu_update(X, idx, C_prev)
+    assert np.array_equal(counts_gpu, counts_or)
+    assert u.centroid_rel_err(C_gpu, C_or, X) <= u.REL_CENTROID
+    p = rng.permutation(len(X))
+    C_perm, _ = u.gpu_update(X[p], idx[p], C_prev)
+    assert np.array_equal(C_perm.view(np.uint32), C_gpu.view(np.uint32))
+
+
+# ------------------------------------------------------------------ Lloyd loop
+
+def _lockstep(X, C0, iters, full_oracle=True, sel=None):
+    """Drive assign/update from the host; at every iteration the oracle gets the GPU's centroids."""
+    u = _u()
+    C = C0.copy()
+    tolerated, trace = 0, []
+    for it in range(iters):
+        idx, dist, obj, nres = u.gpu_assign(X, C)
+        t, o_idx, d1 = u.check_assign_against_oracle(X, C, idx, dist, sel)
+        tolerated += t
+        if sel is None:
+            assert obj == pytest.approx(d1.sum(), rel=u.REL_OBJECTIVE)
+        C_or, counts_or = oracle.update(X, idx, C)          # oracle M-step on the GPU's own indices
+        C_gpu, counts_gpu = u.gpu_update(X, idx, C)
+        assert np.array_equal(counts_gpu, counts_or)
+        assert u.centroid_rel_err(C_gpu, C_or, X) <= u.REL_CENTROID
+        trace.append(obj)
+        C = C_gpu
+    return C, trace, tolerated
+
+
+def _gpu_fit(X, C0, iters, path=0):
+    cc, u = _cc(), _u()
+    N, g = X.shape
+    K = C0.shape[0]
+    c = u.ctx()
+    c.ensure_workspace(N, g, K)
+    cc.cc_set_path(c, path)
+    Xd, C = u.half_dev(X), u.dev(C0)
+    idx = torch.empty(N, dtype=torch.uint16, device="cuda")
+    dist = torch.empty(N, dtype=torch.float32, device="cuda")
+    counts = torch.empty(K, dtype=torch.int32, device="cuda")
+    trace = torch.empty(max(iters, 1), dtype=torch.float64, device="cuda")
+    cc.cc_fit(c, Xd, N, g, K, iters, C, idx, dist, counts, trace)
+    cc.cc_poll_status(c)
+    cc.cc_set_path(c, 0)
+    return C.cpu().numpy(), u.u16_np(idx).astype(np.int32), dist.cpu().numpy(), counts.cpu().numpy(), \
+        trace.cpu().numpy()[:iters]
+
+
+def test_cfg1_lockstep_fit_and_free_run():
+    u = _u()
+    w = wl.WORKLOADS["cfg1_256x512_g4_k256"]
+    W = wl.make_matrix(w.matrices[0])
+    X = oracle.reshape_subvectors(W, w.g)
+    C0 = oracle.init_codebook(X, w.K, w.matrices[0].init_seed)
+    C_lock, trace_lock, tol = _lockstep(X, C0, w.iters)
+    print("cfg1 tolerated near-ties:", tol)
+    C_fit, idx_fit, dist_fit, counts_fit, trace_fit = _gpu_fit(X, C0, w.iters)
+    assert np.array_equal(C_fit.view(np.uint32), C_lock.view(np.uint32))      # cc_fit == the driven loop
+    assert np.array_equal(trace_fit, np.array(trace_lock))
+    assert np.all(np.diff(trace_fit) <= 1e-6 * trace_fit[:-1])                # objective never increases
+    C_or, idx_or, d1_or, counts_or, obj_or = oracle.fit(X, C0, w.iters)        # free-running oracle
+    assert trace_fit[-1] == pytest.approx(obj_or[-1], rel=u.REL_OBJECTIVE)
+    assert np.allclose(trace_fit, obj_or, rtol=u.REL_OBJECTIVE)
+    assert counts_fit.sum() == len(X)
+
+
+def test_blobs_recovered_and_k_equals_n():
+    u = _u()
+    X, labels, centres = wl.make_blobs(12, 300, 4, seed=90, sep=1.0, sigma=0.01)
+    first = np.array([np.flatnonzero(labels == b)[0] for b in range(12)])
+    C, idx, dist, counts, trace = _gpu_fit(X, X[first].astype(np.float32), 4)
+    assert np.array_equal(idx, labels) and np.all(counts == 300)
+    Xd = X.astype(np.float64)
+    for b in range(12):
+        assert np.array_equal(C[b], Xd[labels == b].mean(0).astype(np.float32))
+    Xu = np.unique(wl.make_points(3000, 4, 80), axis=0)
+    N = len(Xu)
+    C0 = oracle.init_codebook(Xu, N, 5)
+    C, idx, dist, counts, trace = _gpu_fit(Xu, C0, 2)
+    assert np.all(trace == 0) and np.all(counts == 1) and np.array_equal(C[idx], Xu.astype(np.float32))
+
+
+def test_finalize_decode_identity_and_compress_host():
+    cc, u = _cc(), _u()
+    w = wl.WORKLOADS["cfg1_256x512_g4_k256"]
+    W = wl.make_matrix(w.matrices[0])
+    d_out, d_in = W.shape
+    for layout in (0, 1):
+        N = cc.cc_num_subvectors(d_out, d_in, w.g, layout)
+        C16 = torch.empty((w.K, w.g), dtype=torch.float16).pin_memory()
+        idx = torch.empty(N, dtype=torch.uint16).pin_memory()
+        trace = torch.empty(w.iters + 1, dtype=torch.float64).pin_memory()
+        What = torch.empty((d_out, d_in), dtype=torch.float16).pin_memory()
+        Wh = torch.from_numpy(W.view(np.int16)).view(torch.float16).pin_memory()
+        cc.cc_compress_host(u.ctx(), Wh, d_out, d_in, w.g, w.K, w.iters, w.matrices[0].init_seed, layout, C16, idx,
+                            trace, What)
+        C16n = C16.numpy()
+        idxn = idx.view(torch.int16).numpy().view(np.uint16).astype(np.int32)
+        Whn = What.numpy()
+        err = ((W.astype(np.float64) - Whn.astype(np.float64)) ** 2).sum()
+        assert err == pytest.approx(trace[-1].item(), rel=1e-6)             # ||W - decode||^2 = objective
+        # the oracle agrees on every piece, given the GPU's stored codebook
+        X = oracle.reshape_subvectors(W, w.g, layout)
+        t, o_idx, d1 = u.check_assign_against_oracle(X, C16n.astype(np.float32), idxn, None)
+        assert np.array_equal(Whn.view(np.uint16), oracle.decode(C16n, idxn, d_out, d_in, layout).view(np.uint16))
+        assert trace[-1].item() == pytest.approx(d1.sum(), rel=u.REL_OBJECTIVE)
+        # free-running oracle from the same start reaches the same objective
+        C0 = oracle.init_codebook(X, w.K, w.matrices[0].init_seed)
+        C_or = oracle.fit(X, C0, w.iters)[0]
+        _, _, _, J_or = oracle.finalize(X, C_or)
+        assert trace[-1].item() == pytest.approx(J_or, rel=u.REL_OBJECTIVE)
+        assert np.array_equal(oracle.to_half(C_or).view(np.uint16), C16n.view(np.uint16)) or \
+            u.centroid_rel_err(C16n.astype(np.float32), oracle.to_half(C_or).astype(np.float32), X) < 2e-3
+
+
+# ------------------------------------------------------------------ full-size workloads
+
+def test_cfg2_full_size_lockstep_then_free_run():
+    """The benchmark workload at its full size: first iteration checked on every point, the
+    following ones on a seeded sample; free-running objectives compared over 4 iterations."""
+    u = _u()
+    w = wl.WORKLOADS["cfg2_4096x4096_g4_k4096"]
+    W = wl.make_matrix(w.matrices[0])
+    X = oracle.reshape_subvectors(W, w.g)
+    N = len(X)
+    C0 = oracle.init_codebook(X, w.K, w.matrices[0].init_seed)
+    C1, trace1, tol1 = _lockstep(X, C0, 1)
+    sel = wl.subset_positions(N, 0.02, 77)
+    C3, trace3, tol3 = _lockstep(X, C1, 2, sel=sel)
+    print("cfg2 tolerated near-ties: full %d, sampled %d" % (tol1, tol3))
+    C_fit, idx_fit, dist_fit, counts_fit, trace_fit = _gpu_fit(X, C0, 4)
+    obj_or = oracle.fit(X, C0, 4)[4]
+    assert np.allclose(trace_fit, obj_or, rtol=u.REL_OBJECTIVE)
+    assert np.array_equal(trace_fit[:3], np.array(trace1 + trace3))
+
+
+@pytest.mark.parametrize("name,mat,frac", [("cfg3_4096x11008_g8_k65536", 0, 0.0008),
+                                           ("cfg5_layer7b_g16_k65536", 0, 0.002),
+                                           ("cfg5_layer7b_g16_k65536", 6, 0.0008)])
+def test_large_k_workloads_sampled(name, mat, frac):
+    """K = 65536 at full N: two iterations, the oracle checks a seeded sample of the points
+    against all centroids and runs its M-step on all points."""
+    u = _u()
+    w = wl.WORKLOADS[name]
+    spec = w.matrices[mat]
+    X = oracle.reshape_subvectors(wl.make_matrix(spec), w.g)
+    C0 = oracle.init_codebook(X, w.K, spec.init_seed)
+    sel = wl.subset_positions(len(X), frac, 5)
+    C, trace, tol = _lockstep(X, C0, 2, sel=sel)
+    print(name, spec.name, "tolerated near-ties on the sample:", tol, "objective", trace)
+    assert trace[1] < trace[0]
+
+
+def test_cfg4_full_size_one_iteration_sampled():
+    u = _u()
+    w = wl.WORKLOADS["cfg4_8192x28672_g4_k65536"]
+    spec = w.matrices[0]
+    X = oracle.reshape_subvectors(wl.make_matrix(spec), w.g)
+    C0 = oracle.init_codebook(X, w.K, spec.init_seed)
+    sel = wl.subset_positions(len(X), 0.0002, 5)
+    C, trace, tol = _lockstep(X, C0, 1, sel=sel)
+    print("cfg4 tolerated near-ties on the sample:", tol, "objective", trace)

@@ -4,9 +4,9 @@
 // Fast stage.  For point x and centroid c the comparison score is
 //     s = ||c||^2 - 2 x.c        (||x||^2 is the same for every centroid and dropped)
 // computed as one FMA chain  s = fma(x_{g-1}, m_{g-1}, ... fma(x_0, m_0, csq))  with m = -2c and
-// csq = ||c||^2 staged once per call.  Each thread keeps P points in registers (as f32x2 pairs of
-// two points) and walks the staged codebook through shared memory; every shared-memory value is
-// read by the whole warp at once (a broadcast).  Only the running MINIMUM of the scores is kept
+// csq = ||c||^2 staged once per call.  Each thread keeps P points in registers and walks the staged
+// codebook through shared memory; every shared-memory value is read by the whole warp at once (a
+// broadcast).  For g <= 4 the FMAs are the packed two-wide form over pairs of centroids.  Only the running MINIMUM of the scores is kept
 // in the inner loop (one 3-input min per two scores); the minimum is tracked per chunk of CHUNK
 // centroids, together with the best and second-best chunk minima, and the winning chunk is
 // rescanned once per point at the end to recover the index and the runner-up inside it.
@@ -53,11 +53,18 @@ __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wai
 constexpr float kBig = 3.0e38f;   // score of the padding centroids; above any real score
 constexpr int kThreads = 256;
 
+// Per-g tiling.  PACKED: two-wide FMAs over pairs of centroids (each point's coordinates are held
+// twice in a 64-bit register pair); otherwise scalar FMAs and twice as many points per thread.
+// Either way a thread's points cost at most 64 registers.  A shared-memory load is a broadcast,
+// but it still returns 512 bytes per warp, so the number of points per thread is what keeps the
+// load pipe below the FMA pipes.
 template <int G> struct FfmaCfg {
-    static constexpr int P = (G <= 8) ? 8 : 4;                       // points per thread
-    static constexpr int TILE = (G <= 4) ? 512 : (G <= 8) ? 256 : 128;  // centroids per smem tile
-    static constexpr int CHUNK = 32;                                  // centroids per tracked minimum
-    static constexpr int ROW4 = G + 1;                                // float4 per centroid pair
+    static constexpr bool PACKED = (G <= 4);
+    static constexpr int P_RAW = PACKED ? 32 / G : 64 / G;
+    static constexpr int P = P_RAW > 16 ? 16 : (P_RAW < 4 ? 4 : (P_RAW & ~1));   // points per thread
+    static constexpr int TILE = (G <= 4) ? 1024 : (G <= 8) ? 512 : 256;          // centroids per smem tile
+    static constexpr int CHUNK = 32;                                             // centroids per tracked minimum
+    static constexpr int ROW4 = G + 1;                                           // float4 per 4 centroids
 };
 
 // Load one point (G halves) as floats; rows beyond N read as zeros.
@@ -102,10 +109,9 @@ __device__ __forceinline__ void load_point(const uint16_t* __restrict__ X, int64
     }
 }
 
-// Staged codebook: for each pair of centroids (2q, 2q+1), G float4 {m_{2q,t}, m_{2q,t}, m_{2q+1,t},
-// m_{2q+1,t}} followed by {csq_{2q}, csq_{2q}, csq_{2q+1}, csq_{2q+1}}; m = -2c.  Each value appears
-// twice so that one 128-bit shared load yields two ready f32x2 operands (one per centroid, the same
-// value for both points of a pair).  Centroids K..Kpad-1 are padding that can never win.
+// Staged codebook: for each group of four centroids j..j+3, G float4 {m_{j,t} .. m_{j+3,t}}
+// (t = 0..G-1, m = -2c) followed by {csq_j .. csq_{j+3}}.  Centroids K..Kpad-1 are padding that
+// can never win.
 template <int G>
 __global__ void prep_ffma_kernel(const float* __restrict__ C, int K, int Kpad, float4* __restrict__ prep,
                                  unsigned* __restrict__ status) {
@@ -113,11 +119,11 @@ __global__ void prep_ffma_kernel(const float* __restrict__ C, int K, int Kpad, f
     if (q == 0) {  // reset the flagged-point counter of this E-step
         *reinterpret_cast<ull*>(status + 2) = 0ull;
     }
-    if (q >= Kpad / 2) return;
-    float m[2][G], csq[2];
+    if (q >= Kpad / 4) return;
+    float m[4][G], csq[4];
 #pragma unroll
-    for (int h = 0; h < 2; ++h) {
-        int j = 2 * q + h;
+    for (int h = 0; h < 4; ++h) {
+        int j = 4 * q + h;
         if (j < K) {
             double s = 0.0;
 #pragma unroll
@@ -135,35 +141,41 @@ __global__ void prep_ffma_kernel(const float* __restrict__ C, int K, int Kpad, f
     }
     float4* out = prep + (int64_t)q * (G + 1);
 #pragma unroll
-    for (int t = 0; t < G; ++t) out[t] = make_float4(m[0][t], m[0][t], m[1][t], m[1][t]);
-    out[G] = make_float4(csq[0], csq[0], csq[1], csq[1]);
+    for (int t = 0; t < G; ++t) out[t] = make_float4(m[0][t], m[1][t], m[2][t], m[3][t]);
+    out[G] = make_float4(csq[0], csq[1], csq[2], csq[3]);
 }
 
 template <int G>
-__global__ void __launch_bounds__(kThreads, (G <= 4) ? 2 : 1)
+__global__ void __launch_bounds__(kThreads, 1)
 assign_ffma_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restrict__ C, int K, int Kpad,
                    const float4* __restrict__ prep, uint16_t* __restrict__ idx, float* __restrict__ dist,
                    unsigned* __restrict__ status, unsigned* __restrict__ flagged) {
     using Cfg = FfmaCfg<G>;
     constexpr int P = Cfg::P, TILE = Cfg::TILE, CHUNK = Cfg::CHUNK, ROW4 = Cfg::ROW4;
-    constexpr int TILE4 = TILE / 2 * ROW4;   // float4 per tile
-    static_assert(P * kThreads * 2 * 4 <= 2 * TILE4 * 16, "stash must fit in the tile buffers");
-    __shared__ float4 tiles[2][TILE4];
+    constexpr bool PACKED = Cfg::PACKED;
+    constexpr int TILE4 = TILE / 4 * ROW4;   // float4 per tile
+    constexpr int STASH4 = P * kThreads * 2 * 4 / 32;   // float4 per buffer needed by the final stash
+    constexpr int BUF4 = TILE4 > STASH4 ? TILE4 : STASH4;
+    static_assert(2 * BUF4 * 16 <= 48 * 1024, "static shared memory limit");
+    __shared__ float4 tiles[2][BUF4];
 
     const int tid = threadIdx.x;
     const int64_t base = (int64_t)blockIdx.x * (kThreads * P);
 
-    // ---- points of this thread, as pairs (point 2pp, point 2pp+1) per dimension
-    ull xp[P / 2][G];
+    // ---- points of this thread: point p is row base + p*kThreads + tid
+    constexpr int XW = PACKED ? 2 : 1;
+    float xs[P][G];          // scalar mode operands (also the source of the packed copies)
+    ull xd[PACKED ? P : 1][PACKED ? G : 1];
     bool nonfinite = false;
 #pragma unroll
-    for (int pp = 0; pp < P / 2; ++pp) {
-        float xa[G], xb[G];
-        load_point<G>(X, base + (int64_t)(2 * pp) * kThreads + tid, N, xa, nonfinite);
-        load_point<G>(X, base + (int64_t)(2 * pp + 1) * kThreads + tid, N, xb, nonfinite);
+    for (int p = 0; p < P; ++p) {
+        load_point<G>(X, base + (int64_t)p * kThreads + tid, N, xs[p], nonfinite);
+        if constexpr (PACKED) {
 #pragma unroll
-        for (int t = 0; t < G; ++t) xp[pp][t] = pack2(xa[t], xb[t]);
+            for (int t = 0; t < G; ++t) xd[p][t] = pack2(xs[p][t], xs[p][t]);
+        }
     }
+    (void)XW;
     if (nonfinite) atomicOr(status, CC_DEV_NONFINITE);
 
     float b1[P], b2[P];
@@ -172,7 +184,6 @@ assign_ffma_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __res
     for (int p = 0; p < P; ++p) { b1[p] = INFINITY; b2[p] = INFINITY; bc[p] = 0; }
 
     const int n_tiles = Kpad / TILE;
-    // prefetch tile 0
     for (int e = tid; e < TILE4; e += kThreads) cp_async16(&tiles[0][e], prep + e);
     cp_async_commit();
 
@@ -191,30 +202,54 @@ assign_ffma_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __res
             float m[P];
 #pragma unroll
             for (int p = 0; p < P; ++p) m[p] = INFINITY;
-            const float4* cp = tbuf + c * (CHUNK / 2) * ROW4;
+            const float4* cp = tbuf + c * (CHUNK / 4) * ROW4;
 #pragma unroll 2
-            for (int q = 0; q < CHUNK / 2; ++q) {
+            for (int q = 0; q < CHUNK / 4; ++q) {
                 const float4* row = cp + q * ROW4;
-                float4 cs = row[G];
-                ull accA[P / 2], accB[P / 2];
-                const ull csA = pack2(cs.x, cs.y), csB = pack2(cs.z, cs.w);
+                const float4 cs = row[G];
+                if constexpr (PACKED) {
+                    ull lo[P], hi[P];
+                    const ull csLo = pack2(cs.x, cs.y), csHi = pack2(cs.z, cs.w);
 #pragma unroll
-                for (int t = 0; t < G; ++t) {
-                    float4 mv = row[t];
-                    const ull mA = pack2(mv.x, mv.y), mB = pack2(mv.z, mv.w);
+                    for (int t = 0; t < G; ++t) {
+                        const float4 mv = row[t];
+                        const ull mLo = pack2(mv.x, mv.y), mHi = pack2(mv.z, mv.w);
 #pragma unroll
-                    for (int pp = 0; pp < P / 2; ++pp) {
-                        accA[pp] = fma2(xp[pp][t], mA, t == 0 ? csA : accA[pp]);
-                        accB[pp] = fma2(xp[pp][t], mB, t == 0 ? csB : accB[pp]);
+                        for (int p = 0; p < P; ++p) {
+                            lo[p] = fma2(xd[p][t], mLo, t == 0 ? csLo : lo[p]);
+                            hi[p] = fma2(xd[p][t], mHi, t == 0 ? csHi : hi[p]);
+                        }
                     }
-                }
 #pragma unroll
-                for (int pp = 0; pp < P / 2; ++pp) {
-                    float a0, a1, c0, c1;
-                    unpack2(accA[pp], a0, a1);
-                    unpack2(accB[pp], c0, c1);
-                    m[2 * pp] = min3(m[2 * pp], a0, c0);
-                    m[2 * pp + 1] = min3(m[2 * pp + 1], a1, c1);
+                    for (int p = 0; p < P; ++p) {
+                        float a0, a1, c0, c1;
+                        unpack2(lo[p], a0, a1);
+                        unpack2(hi[p], c0, c1);
+                        m[p] = min3(m[p], a0, a1);
+                        m[p] = min3(m[p], c0, c1);
+                    }
+                } else {
+                    float mv[G][4];
+#pragma unroll
+                    for (int t = 0; t < G; ++t) {
+                        const float4 v = row[t];
+                        mv[t][0] = v.x; mv[t][1] = v.y; mv[t][2] = v.z; mv[t][3] = v.w;
+                    }
+                    const float csv[4] = {cs.x, cs.y, cs.z, cs.w};
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {          // two centroids at a time
+                        float a0[P], a1[P];
+#pragma unroll
+                        for (int t = 0; t < G; ++t) {
+#pragma unroll
+                            for (int p = 0; p < P; ++p) {
+                                a0[p] = fmaf(xs[p][t], mv[t][2 * h], t == 0 ? csv[2 * h] : a0[p]);
+                                a1[p] = fmaf(xs[p][t], mv[t][2 * h + 1], t == 0 ? csv[2 * h + 1] : a1[p]);
+                            }
+                        }
+#pragma unroll
+                        for (int p = 0; p < P; ++p) m[p] = min3(m[p], a0[p], a1[p]);
+                    }
                 }
             }
             const int chunk_id = tile * (TILE / CHUNK) + c;
@@ -250,21 +285,25 @@ assign_ffma_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __res
         // rescan the winning chunk: same FMA chain, ascending j, strict '<' keeps the lowest index
         float s1 = INFINITY, s2 = INFINITY;
         int j1 = chunk * CHUNK;
-        const float4* cp = prep + (int64_t)chunk * (CHUNK / 2) * ROW4;
-#pragma unroll 2
-        for (int q = 0; q < CHUNK / 2; ++q) {
+        const float4* cp = prep + (int64_t)chunk * (CHUNK / 4) * ROW4;
+#pragma unroll 1
+        for (int q = 0; q < CHUNK / 4; ++q) {
             const float4* row = cp + q * ROW4;
-            float4 cs = __ldg(row + G);
-            float sa = cs.x, sb = cs.z;
+            const float4 cs = __ldg(row + G);
+            float s[4] = {cs.x, cs.y, cs.z, cs.w};
 #pragma unroll
             for (int t = 0; t < G; ++t) {
-                float4 mv = __ldg(row + t);
-                sa = fmaf(x[t], mv.x, sa);
-                sb = fmaf(x[t], mv.z, sb);
+                const float4 mv = __ldg(row + t);
+                s[0] = fmaf(x[t], mv.x, s[0]);
+                s[1] = fmaf(x[t], mv.y, s[1]);
+                s[2] = fmaf(x[t], mv.z, s[2]);
+                s[3] = fmaf(x[t], mv.w, s[3]);
             }
-            const int j = chunk * CHUNK + 2 * q;
-            if (sa < s1) { s2 = s1; s1 = sa; j1 = j; } else if (sa < s2) s2 = sa;
-            if (sb < s1) { s2 = s1; s1 = sb; j1 = j + 1; } else if (sb < s2) s2 = sb;
+#pragma unroll
+            for (int h = 0; h < 4; ++h) {
+                if (s[h] < s1) { s2 = s1; s1 = s[h]; j1 = chunk * CHUNK + 4 * q + h; }
+                else if (s[h] < s2) s2 = s[h];
+            }
         }
         if (j1 >= K) j1 = K - 1;   // only reachable with non-finite input
         s2 = fminf(s2, second_other);
@@ -272,10 +311,10 @@ assign_ffma_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __res
         double A = 0.0, D = 0.0;
 #pragma unroll
         for (int t = 0; t < G; ++t) {
-            const double xd = (double)x[t];
-            const double df = __dsub_rn(xd, (double)__ldg(C + (int64_t)j1 * G + t));
+            const double xdbl = (double)x[t];
+            const double df = __dsub_rn(xdbl, (double)__ldg(C + (int64_t)j1 * G + t));
             D = __dadd_rn(D, __dmul_rn(df, df));
-            A = __dadd_rn(A, __dmul_rn(xd, xd));
+            A = __dadd_rn(A, __dmul_rn(xdbl, xdbl));
         }
         idx[i] = (uint16_t)j1;
         dist[i] = (float)D;
@@ -288,19 +327,30 @@ assign_ffma_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __res
 }
 
 // ---------------------------------------------------------------------------------------------
-// Exact stage: one thread per flagged point scans every centroid.  A cheap FP32 direct-form
+// Exact stage.  Each flagged point is scanned against every centroid by a group of T lanes of a
+// warp (T = 32, 8 or 1, chosen from the number of flagged points so that few points still fill
+// the GPU and many points do not re-read the codebook too often).  A cheap FP32 direct-form
 // distance (relative error <= (g+2) 2^-24, no cancellation) screens the candidates; those within
 // 2^-18 of the best FP64 distance so far are recomputed in FP64 (sub, mul, add, in dimension
 // order, no FMA contraction) and the pair (distance, index) is minimised lexicographically.
 template <int G>
-__global__ void __launch_bounds__(64)
+__global__ void __launch_bounds__(128)
 resolve_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restrict__ C, int K,
                const unsigned* __restrict__ status, const unsigned* __restrict__ flagged,
                uint16_t* __restrict__ idx, float* __restrict__ dist) {
     ull F = *reinterpret_cast<const ull*>(status + 2);
     if (F > (ull)N) F = (ull)N;
-    for (ull f = (ull)blockIdx.x * blockDim.x + threadIdx.x; f < F; f += (ull)gridDim.x * blockDim.x) {
-        const int64_t i = flagged[f];
+    if (F == 0) return;
+    const ull total_threads = (ull)gridDim.x * blockDim.x;
+    const int T = (F * 32 <= total_threads) ? 32 : (F * 8 <= total_threads) ? 8 : 1;
+    const ull gthread = (ull)blockIdx.x * blockDim.x + threadIdx.x;
+    const int lane = (int)(gthread % T);
+    const ull n_groups = total_threads / T;
+    const ull n_rounds = (F + n_groups - 1) / n_groups;       // the same for every lane of a warp
+    for (ull r = 0; r < n_rounds; ++r) {
+        const ull f = r * n_groups + gthread / T;
+        const bool live = f < F;
+        const int64_t i = live ? flagged[f] : 0;
         float x[G];
         bool nf = false;
         load_point<G>(X, i, N, x, nf);
@@ -312,8 +362,8 @@ resolve_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restric
             Db = __dadd_rn(Db, __dmul_rn(df, df));
         }
         float bound = __double2float_ru(Db * (1.0 + 3.814697265625e-6));
-#pragma unroll 4
-        for (int j = 0; j < K; ++j) {
+#pragma unroll 2
+        for (int j = lane; j < K; j += T) {
             float c[G];
 #pragma unroll
             for (int t = 0; t < G; ++t) c[t] = __ldg(C + (int64_t)j * G + t);
@@ -333,8 +383,16 @@ resolve_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restric
                 }
             }
         }
-        idx[i] = (uint16_t)jb;
-        dist[i] = (float)Db;
+        // lexicographic minimum of (distance, index) over the T lanes of the group
+        for (int o = T >> 1; o > 0; o >>= 1) {
+            const double Do = __shfl_xor_sync(0xffffffffu, Db, o);
+            const int jo = __shfl_xor_sync(0xffffffffu, jb, o);
+            if (Do < Db || (Do == Db && jo < jb)) { Db = Do; jb = jo; }
+        }
+        if (live && lane == 0) {
+            idx[i] = (uint16_t)jb;
+            dist[i] = (float)Db;
+        }
     }
 }
 
@@ -390,7 +448,7 @@ cudaError_t launch_ffma(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64
     const int Kpad = (int)cc_align_up((size_t)K, CC_KPAD);
     {
         ProfScope ps(ctx, CC_K_ASSIGN_PREP, st);
-        prep_ffma_kernel<G><<<(Kpad / 2 + 127) / 128, 128, 0, st>>>(C, K, Kpad, prep, status);
+        prep_ffma_kernel<G><<<(Kpad / 4 + 127) / 128, 128, 0, st>>>(C, K, Kpad, prep, status);
     }
     if (N > 0) {
         const int64_t per_block = (int64_t)kThreads * FfmaCfg<G>::P;
@@ -411,7 +469,7 @@ cudaError_t launch_tail(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64
     double* partials = reinterpret_cast<double*>(ws + L.partials);
     if (N > 0) {
         ProfScope ps(ctx, CC_K_RESOLVE, st);
-        resolve_kernel<G><<<ctx->sm_count * 8, 64, 0, st>>>(X, N, C, K, status, flagged, idx, dist);
+        resolve_kernel<G><<<ctx->sm_count * 16, 128, 0, st>>>(X, N, C, K, status, flagged, idx, dist);
     }
     if (objective || n_resolved) {
         int blocks = (int)((N + 4095) / 4096);

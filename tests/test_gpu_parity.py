@@ -90,10 +90,10 @@ def test_assign_exact_ties_and_duplicates_take_lowest_index():
     g, K, N = 4, 600, 4000
     X = wl.make_points(N, g, 5)
     C = wl.make_codebook(K, g, 6)
-    C[300:400] = C[100:200]                       # duplicated centroids
-    C[450] = C[3]
     X[:K] = C.astype(np.float16)                  # points sitting (almost) on centroids
     C[:64] = X[:64].astype(np.float32)            # ... and exactly on them
+    C[300:400] = C[100:200]                       # duplicated centroids
+    C[450] = C[3]
     idx, dist, obj, nres = u.gpu_assign(X, C)
     o_idx, d1, d2 = oracle.assign(X, C)
     assert np.array_equal(idx, o_idx)             # exact ties included: no tolerance here

@@ -65,6 +65,7 @@ template <int G> struct FfmaCfg {
     static constexpr int TILE = (G <= 4) ? 1024 : (G <= 8) ? 512 : 256;          // centroids per smem tile
     static constexpr int CHUNK = 32;                                             // centroids per tracked minimum
     static constexpr int ROW4 = G + 1;                                           // float4 per 4 centroids
+    static constexpr int MIN_BLOCKS = (G <= 4) ? 2 : 1;                          // resident blocks per SM aimed at
 };
 
 // Load one point (G halves) as floats; rows beyond N read as zeros.
@@ -146,7 +147,7 @@ __global__ void prep_ffma_kernel(const float* __restrict__ C, int K, int Kpad, f
 }
 
 template <int G>
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, FfmaCfg<G>::MIN_BLOCKS)
 assign_ffma_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restrict__ C, int K, int Kpad,
                    const float4* __restrict__ prep, uint16_t* __restrict__ idx, float* __restrict__ dist,
                    unsigned* __restrict__ status, unsigned* __restrict__ flagged) {
@@ -208,25 +209,25 @@ assign_ffma_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __res
                 const float4* row = cp + q * ROW4;
                 const float4 cs = row[G];
                 if constexpr (PACKED) {
-                    ull lo[P], hi[P];
-                    const ull csLo = pack2(cs.x, cs.y), csHi = pack2(cs.z, cs.w);
+                    float4 mv[G];
 #pragma unroll
-                    for (int t = 0; t < G; ++t) {
-                        const float4 mv = row[t];
-                        const ull mLo = pack2(mv.x, mv.y), mHi = pack2(mv.z, mv.w);
+                    for (int t = 0; t < G; ++t) mv[t] = row[t];
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {          // centroids (j, j+1), then (j+2, j+3)
+                        ull acc[P];
+                        const ull cs2 = h ? pack2(cs.z, cs.w) : pack2(cs.x, cs.y);
+#pragma unroll
+                        for (int t = 0; t < G; ++t) {
+                            const ull m2 = h ? pack2(mv[t].z, mv[t].w) : pack2(mv[t].x, mv[t].y);
+#pragma unroll
+                            for (int p = 0; p < P; ++p) acc[p] = fma2(xd[p][t], m2, t == 0 ? cs2 : acc[p]);
+                        }
 #pragma unroll
                         for (int p = 0; p < P; ++p) {
-                            lo[p] = fma2(xd[p][t], mLo, t == 0 ? csLo : lo[p]);
-                            hi[p] = fma2(xd[p][t], mHi, t == 0 ? csHi : hi[p]);
+                            float a0, a1;
+                            unpack2(acc[p], a0, a1);
+                            m[p] = min3(m[p], a0, a1);
                         }
-                    }
-#pragma unroll
-                    for (int p = 0; p < P; ++p) {
-                        float a0, a1, c0, c1;
-                        unpack2(lo[p], a0, a1);
-                        unpack2(hi[p], c0, c1);
-                        m[p] = min3(m[p], a0, a1);
-                        m[p] = min3(m[p], c0, c1);
                     }
                 } else {
                     float mv[G][4];
@@ -286,7 +287,7 @@ assign_ffma_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __res
         float s1 = INFINITY, s2 = INFINITY;
         int j1 = chunk * CHUNK;
         const float4* cp = prep + (int64_t)chunk * (CHUNK / 4) * ROW4;
-#pragma unroll 1
+#pragma unroll
         for (int q = 0; q < CHUNK / 4; ++q) {
             const float4* row = cp + q * ROW4;
             const float4 cs = __ldg(row + G);
@@ -362,8 +363,9 @@ resolve_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restric
             Db = __dadd_rn(Db, __dmul_rn(df, df));
         }
         float bound = __double2float_ru(Db * (1.0 + 3.814697265625e-6));
+        const int k_end = live ? K : 0;        // idle groups skip the scan
 #pragma unroll 2
-        for (int j = lane; j < K; j += T) {
+        for (int j = lane; j < k_end; j += T) {
             float c[G];
 #pragma unroll
             for (int t = 0; t < G; ++t) c[t] = __ldg(C + (int64_t)j * G + t);

@@ -98,7 +98,8 @@ int64_t cc_launch_count(const cc_ctx* ctx);
 #define CC_KERNEL_RESHAPE 6
 #define CC_KERNEL_DECODE 7
 #define CC_KERNEL_OTHER 8
-#define CC_KERNEL_CLASSES 9
+#define CC_KERNEL_ASSIGN_FINISH 9 /* tensor path: index, distance, near-tie flag per point */
+#define CC_KERNEL_CLASSES 10
 cc_status cc_profile_enable(cc_ctx* ctx, int on);
 cc_status cc_profile_read(cc_ctx* ctx, double* total_ms_host, int64_t* launches_host);
 

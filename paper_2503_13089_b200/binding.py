@@ -149,7 +149,7 @@ def cc_launch_count(ctx: Context) -> int:
 
 
 KERNEL_CLASSES = ("assign_main", "assign_prep", "resolve", "objective", "update_accum", "update_finish",
-                  "reshape", "decode", "other")
+                  "reshape", "decode", "other", "assign_finish")
 
 
 def cc_profile_enable(ctx: Context, on: bool) -> None:

@@ -23,6 +23,7 @@ WsLayout cc_ws_layout(int64_t N, int g, int K) {
     L.dist_tmp = take((size_t)N * 4);
     // tensor-core staging: split codebook operand (Kpad x 64 floats at most) + squared norms
     L.tensor = take(Kpad * (size_t)(64 + 1) * 4);
+    L.tstate = take((size_t)N * 8);
     L.total = off;
     return L;
 }

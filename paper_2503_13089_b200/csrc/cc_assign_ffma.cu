@@ -19,10 +19,9 @@
 #include <float.h>
 
 #include "cc_common.cuh"
+#include "cc_assign_shared.cuh"
 
 namespace {
-
-typedef unsigned long long ull;
 
 __device__ __forceinline__ ull pack2(float lo, float hi) {
     ull r;
@@ -50,7 +49,6 @@ __device__ __forceinline__ void cp_async16(void* smem, const void* gmem) {
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;"); }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 
-constexpr float kBig = 3.0e38f;   // score of the padding centroids; above any real score
 constexpr int kThreads = 256;
 
 // Per-g tiling.  PACKED: two-wide FMAs over pairs of centroids (each point's coordinates are held
@@ -67,48 +65,6 @@ template <int G> struct FfmaCfg {
     static constexpr int ROW4 = G + 1;                                           // float4 per 4 centroids
     static constexpr int MIN_BLOCKS = (G <= 4) ? 2 : 1;                          // resident blocks per SM aimed at
 };
-
-// Load one point (G halves) as floats; rows beyond N read as zeros.
-template <int G>
-__device__ __forceinline__ void load_point(const uint16_t* __restrict__ X, int64_t i, int64_t N, float* x,
-                                           bool& nonfinite) {
-    if (i >= N) {
-#pragma unroll
-        for (int t = 0; t < G; ++t) x[t] = 0.f;
-        return;
-    }
-    const uint16_t* row = X + i * G;
-    uint16_t h[G];
-    if constexpr (G % 8 == 0) {
-#pragma unroll
-        for (int v = 0; v < G / 8; ++v) {
-            uint4 u = __ldg(reinterpret_cast<const uint4*>(row) + v);
-            unsigned w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-            for (int k = 0; k < 4; ++k) { h[v * 8 + 2 * k] = w[k] & 0xffffu; h[v * 8 + 2 * k + 1] = w[k] >> 16; }
-        }
-    } else if constexpr (G % 4 == 0) {
-#pragma unroll
-        for (int v = 0; v < G / 4; ++v) {
-            uint2 u = __ldg(reinterpret_cast<const uint2*>(row) + v);
-            h[v * 4] = u.x & 0xffffu; h[v * 4 + 1] = u.x >> 16; h[v * 4 + 2] = u.y & 0xffffu; h[v * 4 + 3] = u.y >> 16;
-        }
-    } else if constexpr (G % 2 == 0) {
-#pragma unroll
-        for (int v = 0; v < G / 2; ++v) {
-            unsigned u = __ldg(reinterpret_cast<const unsigned*>(row) + v);
-            h[v * 2] = u & 0xffffu; h[v * 2 + 1] = u >> 16;
-        }
-    } else {
-#pragma unroll
-        for (int t = 0; t < G; ++t) h[t] = __ldg(row + t);
-    }
-#pragma unroll
-    for (int t = 0; t < G; ++t) {
-        if ((h[t] & 0x7c00u) == 0x7c00u) nonfinite = true;
-        x[t] = __half2float(__ushort_as_half(h[t]));
-    }
-}
 
 // Staged codebook: for each group of four centroids j..j+3, G float4 {m_{j,t} .. m_{j+3,t}}
 // (t = 0..G-1, m = -2c) followed by {csq_j .. csq_{j+3}}.  Centroids K..Kpad-1 are padding that
@@ -273,57 +229,13 @@ assign_ffma_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __res
     }
     // (each thread reads back only what it wrote: no barrier needed)
 
-    constexpr double kErr = 2.0 * (G + 2) * 5.9604644775390625e-8;   // 2 * gamma_{g+1}, with margin
 #pragma unroll 1
     for (int p = 0; p < P; ++p) {
         const int64_t i = base + (int64_t)p * kThreads + tid;
         if (i >= N) continue;
         const float second_other = stash[(0 * P + p) * kThreads + tid];
         const int chunk = __float_as_int(stash[(1 * P + p) * kThreads + tid]);
-        float x[G];
-        bool nf = false;
-        load_point<G>(X, i, N, x, nf);
-        // rescan the winning chunk: same FMA chain, ascending j, strict '<' keeps the lowest index
-        float s1 = INFINITY, s2 = INFINITY;
-        int j1 = chunk * CHUNK;
-        const float4* cp = prep + (int64_t)chunk * (CHUNK / 4) * ROW4;
-#pragma unroll
-        for (int q = 0; q < CHUNK / 4; ++q) {
-            const float4* row = cp + q * ROW4;
-            const float4 cs = __ldg(row + G);
-            float s[4] = {cs.x, cs.y, cs.z, cs.w};
-#pragma unroll
-            for (int t = 0; t < G; ++t) {
-                const float4 mv = __ldg(row + t);
-                s[0] = fmaf(x[t], mv.x, s[0]);
-                s[1] = fmaf(x[t], mv.y, s[1]);
-                s[2] = fmaf(x[t], mv.z, s[2]);
-                s[3] = fmaf(x[t], mv.w, s[3]);
-            }
-#pragma unroll
-            for (int h = 0; h < 4; ++h) {
-                if (s[h] < s1) { s2 = s1; s1 = s[h]; j1 = chunk * CHUNK + 4 * q + h; }
-                else if (s[h] < s2) s2 = s[h];
-            }
-        }
-        if (j1 >= K) j1 = K - 1;   // only reachable with non-finite input
-        s2 = fminf(s2, second_other);
-        // squared distance to the winner, direct form in FP64 (no contraction)
-        double A = 0.0, D = 0.0;
-#pragma unroll
-        for (int t = 0; t < G; ++t) {
-            const double xdbl = (double)x[t];
-            const double df = __dsub_rn(xdbl, (double)__ldg(C + (int64_t)j1 * G + t));
-            D = __dadd_rn(D, __dmul_rn(df, df));
-            A = __dadd_rn(A, __dmul_rn(xdbl, xdbl));
-        }
-        idx[i] = (uint16_t)j1;
-        dist[i] = (float)D;
-        const double gap = (double)s2 - (double)s1;
-        if (!(gap > kErr * (5.0 * A + 4.0 * D))) {
-            const ull slot = atomicAdd(reinterpret_cast<ull*>(status + 2), 1ull);
-            flagged[slot] = (unsigned)i;
-        }
+        finish_point<G, CHUNK>(X, N, C, K, prep, i, chunk, second_other, (double)(G + 2), idx, dist, status, flagged);
     }
 }
 
@@ -441,6 +353,9 @@ objective_final_kernel(const double* __restrict__ partials, int n, const unsigne
 }
 
 template <int G>
+cudaError_t launch_prep(cc_ctx* ctx, const WsLayout& L, const float* C, int K, cudaStream_t st);
+
+template <int G>
 cudaError_t launch_ffma(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64_t N, const float* C, int K,
                         uint16_t* idx, float* dist, cudaStream_t st) {
     char* ws = static_cast<char*>(ctx->ws);
@@ -448,10 +363,7 @@ cudaError_t launch_ffma(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64
     float4* prep = reinterpret_cast<float4*>(ws + L.cprep);
     unsigned* flagged = reinterpret_cast<unsigned*>(ws + L.flagged);
     const int Kpad = (int)cc_align_up((size_t)K, CC_KPAD);
-    {
-        ProfScope ps(ctx, CC_K_ASSIGN_PREP, st);
-        prep_ffma_kernel<G><<<(Kpad / 4 + 127) / 128, 128, 0, st>>>(C, K, Kpad, prep, status);
-    }
+    launch_prep<G>(ctx, L, C, K, st);
     if (N > 0) {
         const int64_t per_block = (int64_t)kThreads * FfmaCfg<G>::P;
         const int64_t blocks = (N + per_block - 1) / per_block;
@@ -483,6 +395,16 @@ cudaError_t launch_tail(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64
         ProfScope ps(ctx, CC_K_OBJECTIVE, st);
         objective_final_kernel<<<1, 256, 0, st>>>(partials, blocks, status, objective, n_resolved);
     }
+    return cudaGetLastError();
+}
+
+template <int G>
+cudaError_t launch_prep(cc_ctx* ctx, const WsLayout& L, const float* C, int K, cudaStream_t st) {
+    char* ws = static_cast<char*>(ctx->ws);
+    const int Kpad = (int)cc_align_up((size_t)K, CC_KPAD);
+    ProfScope ps(ctx, CC_K_ASSIGN_PREP, st);
+    prep_ffma_kernel<G><<<(Kpad / 4 + 127) / 128, 128, 0, st>>>(C, K, Kpad, reinterpret_cast<float4*>(ws + L.cprep),
+                                                                reinterpret_cast<unsigned*>(ws + L.status));
     return cudaGetLastError();
 }
 
@@ -518,4 +440,12 @@ cudaError_t cc_launch_assign_ffma(cc_ctx* ctx, const WsLayout& L, const uint16_t
 #undef CALL
     if (e != cudaSuccess) return e;
     return cc_launch_assign_tail(ctx, L, X, N, g, C, K, idx, dist, objective, n_resolved, st);
+}
+
+cudaError_t cc_launch_prep_ffma(cc_ctx* ctx, const WsLayout& L, int g, const float* C, int K, cudaStream_t st) {
+    cudaError_t e = cudaSuccess;
+#define CALL(G) e = launch_prep<G>(ctx, L, C, K, st)
+    CC_DISPATCH_G(g, CALL)
+#undef CALL
+    return e;
 }

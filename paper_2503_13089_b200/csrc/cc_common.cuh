@@ -13,7 +13,7 @@
 
 // Kernel classes for the optional per-kernel event timing (cc_profile_*).
 enum { CC_K_ASSIGN_MAIN = 0, CC_K_ASSIGN_PREP = 1, CC_K_RESOLVE = 2, CC_K_OBJECTIVE = 3, CC_K_UPDATE_ACCUM = 4,
-       CC_K_UPDATE_FINISH = 5, CC_K_RESHAPE = 6, CC_K_DECODE = 7, CC_K_OTHER = 8, CC_K_COUNT = 9 };
+       CC_K_UPDATE_FINISH = 5, CC_K_RESHAPE = 6, CC_K_DECODE = 7, CC_K_OTHER = 8, CC_K_ASSIGN_FINISH = 9, CC_K_COUNT = 10 };
 constexpr int CC_PROF_CAP = 8192;
 
 struct cc_prof_slot { cudaEvent_t a, b; int kind; };
@@ -62,7 +62,8 @@ struct WsLayout {
     size_t tmp_c;      // float K x g: widened FP16 codebook (finalize)
     size_t positions;  // int64 K: initial positions
     size_t dist_tmp;   // float N: distances when the caller passes dist == NULL
-    size_t tensor;     // staging of the tensor-core E-step
+    size_t tensor;     // staging of the tensor-core E-step (split codebook operand)
+    size_t tstate;     // float2 N: (second-best chunk minimum, best chunk id) from the tensor-core scan
     size_t total;
 };
 
@@ -85,6 +86,7 @@ cudaError_t cc_launch_to_half(cc_ctx*, const float* C, int64_t n, uint16_t* C16,
 cudaError_t cc_launch_assign_ffma(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const float* C,
                                   int K, uint16_t* idx, float* dist, double* objective, int64_t* n_resolved,
                                   cudaStream_t);
+cudaError_t cc_launch_prep_ffma(cc_ctx*, const WsLayout&, int g, const float* C, int K, cudaStream_t);
 bool cc_tensor_path_supported(int g, int K);
 cudaError_t cc_launch_assign_tensor(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const float* C,
                                     int K, uint16_t* idx, float* dist, double* objective, int64_t* n_resolved,

@@ -85,6 +85,25 @@ def test_assign_matches_oracle(N, g, K):
     assert 0 <= nres <= N
 
 
+@pytest.mark.parametrize("N,g,K", [(1, 4, 1), (2049, 4, 33), (70001, 4, 1000), (20000, 4, 4096), (9000, 8, 300),
+                                   (4097, 8, 2049), (6000, 16, 129), (2500, 16, 1500), (1100, 4, 65536)])
+def test_assign_fp32_and_tensor_paths_agree_with_oracle_and_each_other(N, g, K):
+    cc, u = _cc(), _u()
+    X = wl.make_points(N, g, 1000 + N + g)
+    C = wl.make_codebook(K, g, 2000 + K + g)
+    res = {}
+    for path in (cc.PATH_FFMA, cc.PATH_TENSOR):
+        idx, dist, obj, nres = u.gpu_assign(X, C, path=path)
+        tol, o_idx, d1 = u.check_assign_against_oracle(X, C, idx, dist)
+        assert tol <= max(1, N // 1000)
+        res[path] = (idx, dist, obj)
+    a, b = res[cc.PATH_FFMA], res[cc.PATH_TENSOR]
+    differ = np.flatnonzero(a[0] != b[0])
+    assert len(differ) <= max(1, N // 1000)          # only oracle near-ties may differ between the paths
+    same = a[0] == b[0]
+    assert np.array_equal(a[1][same], b[1][same])
+
+
 def test_assign_exact_ties_and_duplicates_take_lowest_index():
     u = _u()
     g, K, N = 4, 600, 4000

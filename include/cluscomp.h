@@ -49,7 +49,8 @@ typedef enum {
     CC_ERR_NONFINITE = 8,      /* Inf / NaN met in the input (reported by cc_poll_status) */
     CC_ERR_DEVICE_TIMEOUT = 9, /* a bounded device-side wait ran out                      */
     CC_ERR_CUDA = 10,          /* a CUDA runtime call failed                              */
-    CC_ERR_LAYOUT = 11         /* unknown layout / path constant                          */
+    CC_ERR_LAYOUT = 11,        /* unknown layout / path constant                          */
+    CC_ERR_STATIC_CAPACITY = 12 /* cc_update_static: K * g above CC_UPDATE_STATIC_MAX_KG  */
 } cc_status;
 
 /* How sub-vectors are cut out of W (d_out x d_in, row-major, as a linear layer stores it). */
@@ -147,6 +148,37 @@ cc_status cc_assign(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const floa
  * counts (out): K x int32.  idx values must be < K. */
 cc_status cc_update(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const uint16_t* idx, int K,
                     float* C, int32_t* counts, void* stream);
+
+/* M-step without any device allocation (the paper has no counterpart: this is a deployment
+ * variant of cc_update, not a step of the method).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits -- a plug-in inside a process
+ * whose device memory is owned by a framework's pool and may not be grown behind its back, a
+ * serving container whose device memory is fully committed at start-up so that a later
+ * allocation would simply fail, or a latency-critical loop that must never reach the allocator
+ * because cudaMalloc and cudaFree may wait for the whole device.  Such callers have no spare
+ * buffer to hand over as a workspace either, so cc_update (which needs one) is closed to them.
+ *
+ * What it does: exactly what cc_update does, with the same results bit for bit, but the integer
+ * sum accumulators live in a fixed array inside the library image (2 * CC_UPDATE_STATIC_MAX_KG
+ * 64-bit words = 4 MiB).  Every GPU on which the library is loaded holds that array until the
+ * process exits, whether or not this function is ever called.  The function takes no context and
+ * calls no cudaMalloc / cudaFree nor any other allocating routine; the caller still provides
+ * X, idx, C and counts exactly as for cc_update, plus the device ordinal (< 64) that owns them.
+ *
+ * Limits and rules
+ *  - K * g must not exceed CC_UPDATE_STATIC_MAX_KG (262144: K = 65536 at g = 4, K = 16384 at
+ *    g = 16); larger problems return CC_ERR_STATIC_CAPACITY and enqueue nothing.
+ *  - The first call on a device looks up the array's device address (once per device, with
+ *    that device made current).  Make that first call before any stream capture begins.
+ *  - All calls on one device share the one array, and it keeps the previous call's contents:
+ *    each call clears the part it uses on `stream` before accumulating.  Two calls whose work
+ *    overlaps on the GPU (different streams, no dependency) race on it and give wrong sums;
+ *    order them on one stream or with events.  The function is not thread-safe for first calls
+ *    issued concurrently from several host threads on the same device. */
+#define CC_UPDATE_STATIC_MAX_KG 262144
+cc_status cc_update_static(int device, const uint16_t* X, int64_t N, int g, const uint16_t* idx, int K,
+                           float* C, int32_t* counts, void* stream);
 
 /* Lloyd loop of Section 3.1: iters x (E-step, M-step), no early stop (the paper runs a fixed
  * 20).  C: in = initial, out = after the last M-step.  idx / dist / counts (out): those of the

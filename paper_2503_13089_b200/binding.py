@@ -23,8 +23,9 @@ PATH_AUTO, PATH_FFMA, PATH_TENSOR = 0, 1, 2
 STATUS_NAMES = {
     0: "CC_OK", 1: "CC_ERR_NULL", 2: "CC_ERR_SHAPE", 3: "CC_ERR_UNSUPPORTED_G", 4: "CC_ERR_K_RANGE",
     5: "CC_ERR_N_LT_K", 6: "CC_ERR_ALIGN", 7: "CC_ERR_WORKSPACE", 8: "CC_ERR_NONFINITE",
-    9: "CC_ERR_DEVICE_TIMEOUT", 10: "CC_ERR_CUDA", 11: "CC_ERR_LAYOUT",
+    9: "CC_ERR_DEVICE_TIMEOUT", 10: "CC_ERR_CUDA", 11: "CC_ERR_LAYOUT", 12: "CC_ERR_STATIC_CAPACITY",
 }
+UPDATE_STATIC_MAX_KG = 262144
 
 # name -> (restype, argtypes); mirrors include/cluscomp.h one to one
 _vp, _i64, _i32, _u64, _sz, _dbl = ct.c_void_p, ct.c_int64, ct.c_int, ct.c_uint64, ct.c_size_t, ct.c_double
@@ -46,6 +47,7 @@ SIGNATURES = {
     "cc_init_codebook": (_i32, [_vp, _vp, _i64, _i32, _i32, _u64, _vp, _vp]),
     "cc_assign": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp]),
     "cc_update": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp]),
+    "cc_update_static": (_i32, [_i32, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp]),
     "cc_fit": (_i32, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "cc_finalize": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp]),
     "cc_decode": (_i32, [_vp, _vp, _i32, _i32, _vp, _i64, _i64, _i32, _vp, _vp]),
@@ -203,6 +205,13 @@ def cc_assign(ctx, X, N, g, C, K, idx, dist=None, objective=None, n_resolved=Non
 def cc_update(ctx, X, N, g, idx, K, C, counts, stream=None) -> None:
     _check(load().cc_update(ctx._h, _ptr(X), N, g, _ptr(idx), K, _ptr(C), _ptr(counts), _stream(stream)),
            "cc_update")
+
+
+def cc_update_static(device, X, N, g, idx, K, C, counts, stream=None) -> None:
+    """cc_update for callers that may not allocate device memory: no context, no workspace; the
+    accumulators are a fixed array inside the library (K * g <= UPDATE_STATIC_MAX_KG)."""
+    _check(load().cc_update_static(device, _ptr(X), N, g, _ptr(idx), K, _ptr(C), _ptr(counts), _stream(stream)),
+           "cc_update_static")
 
 
 def cc_fit(ctx, X, N, g, K, iters, C, idx, dist, counts, objective_trace=None, stream=None) -> None:

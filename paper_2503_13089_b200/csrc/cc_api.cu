@@ -102,6 +102,7 @@ const char* cc_status_string(cc_status s) {
         case CC_ERR_DEVICE_TIMEOUT: return "device-side wait ran out";
         case CC_ERR_CUDA: return "CUDA runtime error";
         case CC_ERR_LAYOUT: return "unknown layout or path";
+        case CC_ERR_STATIC_CAPACITY: return "K * g above the fixed capacity of cc_update_static";
     }
     return "unknown status";
 }

@@ -103,3 +103,73 @@ cudaError_t cc_launch_update(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, 
                                                              reinterpret_cast<long long*>(sum_hi), counts, K, g, C);
     return cudaGetLastError();
 }
+
+// ---------------------------------------------------------------------------------------------
+// M-step for callers that cannot allocate device memory: the integer sums live in a fixed array
+// that is part of the loaded library image instead of a caller-provided workspace.
+namespace {
+
+constexpr int kStaticMaxDevices = 64;
+
+// [0, CC_UPDATE_STATIC_MAX_KG): sums in units of 2^-24; [MAX_KG, 2*MAX_KG): sums in units of 2^-7.
+static __device__ __align__(256) ull g_static_sums[2 * CC_UPDATE_STATIC_MAX_KG];
+
+// Device address of g_static_sums on each device.  In host code the symbol's name is only a
+// handle; the address a kernel may dereference comes from cudaGetSymbolAddress, asked once per
+// device with that device current.
+void* g_static_addr[kStaticMaxDevices] = {};
+
+cudaError_t static_sums_address(int device, ull** out) {
+    if (!g_static_addr[device]) {
+        void* p = nullptr;
+        const cudaError_t e = cudaGetSymbolAddress(&p, g_static_sums);
+        if (e != cudaSuccess) return e;
+        g_static_addr[device] = p;
+    }
+    *out = static_cast<ull*>(g_static_addr[device]);
+    return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" cc_status cc_update_static(int device, const uint16_t* X, int64_t N, int g, const uint16_t* idx, int K,
+                                      float* C, int32_t* counts, void* stream) {
+    if (!C || !counts || (N > 0 && (!X || !idx))) return CC_ERR_NULL;
+    if (g < 1 || g > 16) return CC_ERR_UNSUPPORTED_G;
+    if (K < 1 || K > 65536) return CC_ERR_K_RANGE;
+    if (N < 0 || N >= (int64_t)1 << 31) return CC_ERR_SHAPE;
+    if ((int64_t)K * g > CC_UPDATE_STATIC_MAX_KG) return CC_ERR_STATIC_CAPACITY;
+    if (device < 0 || device >= kStaticMaxDevices) return CC_ERR_SHAPE;
+    if ((reinterpret_cast<uintptr_t>(X) & 15u) || (reinterpret_cast<uintptr_t>(C) & 15u)) return CC_ERR_ALIGN;
+    if (cudaSetDevice(device) != cudaSuccess) return CC_ERR_CUDA;
+    ull* sums = nullptr;
+    if (static_sums_address(device, &sums) != cudaSuccess) return CC_ERR_CUDA;
+    ull* sum_lo = sums;
+    ull* sum_hi = sums + CC_UPDATE_STATIC_MAX_KG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t used = sizeof(ull) * (size_t)K * g;
+    // the array still holds the previous call's sums
+    if (cudaMemsetAsync(sum_lo, 0, used, st) != cudaSuccess) return CC_ERR_CUDA;
+    if (cudaMemsetAsync(sum_hi, 0, used, st) != cudaSuccess) return CC_ERR_CUDA;
+    if (cudaMemsetAsync(counts, 0, sizeof(int32_t) * (size_t)K, st) != cudaSuccess) return CC_ERR_CUDA;
+    if (N > 0) {
+        int sms = 0;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return CC_ERR_CUDA;
+        int64_t blocks = (N + 255) / 256;
+        const int64_t cap = (int64_t)sms * 16;
+        if (blocks > cap) blocks = cap;
+#define CALL(G)                                                                                               \
+    update_accumulate_kernel<G><<<(unsigned)blocks, 256, 0, st>>>(X, N, idx, K, sum_lo, sum_hi, counts)
+        switch (g) {
+            case 1: CALL(1); break;   case 2: CALL(2); break;   case 3: CALL(3); break;   case 4: CALL(4); break;
+            case 5: CALL(5); break;   case 6: CALL(6); break;   case 7: CALL(7); break;   case 8: CALL(8); break;
+            case 9: CALL(9); break;   case 10: CALL(10); break; case 11: CALL(11); break; case 12: CALL(12); break;
+            case 13: CALL(13); break; case 14: CALL(14); break; case 15: CALL(15); break; case 16: CALL(16); break;
+            default: return CC_ERR_UNSUPPORTED_G;
+        }
+#undef CALL
+    }
+    update_finish_kernel<<<(K * g + 255) / 256, 256, 0, st>>>(reinterpret_cast<long long*>(sum_lo),
+                                                             reinterpret_cast<long long*>(sum_hi), counts, K, g, C);
+    return cudaGetLastError() == cudaSuccess ? CC_OK : CC_ERR_CUDA;
+}

@@ -63,7 +63,7 @@ typedef enum {
 /* Which E-step kernel family cc_assign uses. */
 #define CC_PATH_AUTO 0   /* chosen per (g, K) from measurements                        */
 #define CC_PATH_FFMA 1   /* FP32 FMA pipes, register-tiled                             */
-#define CC_PATH_TENSOR 2 /* tcgen05 tensor cores with TMEM accumulators (g = 4, 8, 16) */
+#define CC_PATH_TENSOR 2 /* tcgen05 tensor cores with TMEM accumulators                */
 
 typedef struct cc_ctx cc_ctx; /* opaque; one per device and per concurrent user */
 
@@ -141,6 +141,15 @@ cc_status cc_init_codebook(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, int
  * N = 0 is allowed (objective 0). */
 cc_status cc_assign(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const float* C, int K,
                     uint16_t* idx, float* dist, double* objective, int64_t* n_resolved, void* stream);
+
+/* Verification aid for the tensor-core E-step (no counterpart in the paper): writes the raw
+ * comparison scores s_ij = ||c_j||^2 - 2 x_i.c_j exactly as that path computes them (FP16 operand
+ * pieces, FP32 accumulation in tensor memory), so that a test can check the rounding bound the
+ * near-tie flag relies on.  scores (out): N rows of cc_tensor_scores_ld(K) floats (K rounded up
+ * to the centroid tile; columns >= K hold the padding score).  1 <= N <= 65536. */
+int64_t cc_tensor_scores_ld(int K);
+cc_status cc_tensor_scores(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const float* C, int K,
+                           float* scores, void* stream);
 
 /* M-step of Section 3.1: counts[j] = |{i : idx[i] = j}| (exact), C[j] = mean of those x_i
  * (exact integer sum, one rounding to FP32); a cluster with no member keeps its centroid

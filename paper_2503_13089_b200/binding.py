@@ -46,6 +46,8 @@ SIGNATURES = {
     "cc_init_positions": (_i32, [_i64, _i32, _u64, _vp]),
     "cc_init_codebook": (_i32, [_vp, _vp, _i64, _i32, _i32, _u64, _vp, _vp]),
     "cc_assign": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp]),
+    "cc_tensor_scores_ld": (_i64, [_i32]),
+    "cc_tensor_scores": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp]),
     "cc_update": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp]),
     "cc_update_static": (_i32, [_i32, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp]),
     "cc_fit": (_i32, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
@@ -200,6 +202,15 @@ def cc_init_codebook(ctx, X, N, g, K, seed, C, stream=None) -> None:
 def cc_assign(ctx, X, N, g, C, K, idx, dist=None, objective=None, n_resolved=None, stream=None) -> None:
     _check(load().cc_assign(ctx._h, _ptr(X), N, g, _ptr(C), K, _ptr(idx), _ptr(dist), _ptr(objective),
                             _ptr(n_resolved), _stream(stream)), "cc_assign")
+
+
+def cc_tensor_scores_ld(K: int) -> int:
+    return int(load().cc_tensor_scores_ld(K))
+
+
+def cc_tensor_scores(ctx, X, N, g, C, K, scores, stream=None) -> None:
+    _check(load().cc_tensor_scores(ctx._h, _ptr(X), N, g, _ptr(C), K, _ptr(scores), _stream(stream)),
+           "cc_tensor_scores")
 
 
 def cc_update(ctx, X, N, g, idx, K, C, counts, stream=None) -> None:

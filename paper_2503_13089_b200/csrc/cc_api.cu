@@ -21,7 +21,8 @@ WsLayout cc_ws_layout(int64_t N, int g, int K) {
     L.tmp_c = take((size_t)K * g * 4);
     L.positions = take((size_t)K * 8);
     L.dist_tmp = take((size_t)N * 4);
-    // tensor-core staging: split codebook operand (Kpad x 64 floats at most) + squared norms
+    // tensor-core staging: FP16 operand image (at most 96 bytes per centroid) followed by the FP32
+    // rows of the finish kernel (at most 68 bytes per centroid)
     L.tensor = take(Kpad * (size_t)(64 + 1) * 4);
     L.tstate = take((size_t)N * 8);
     L.total = off;
@@ -238,6 +239,20 @@ cc_status cc_assign(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const floa
     if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
     const WsLayout L = cc_ws_layout(N, g, K);
     return from_cuda(assign_any(ctx, L, X, N, g, C, K, idx, dist, objective, n_resolved, (cudaStream_t)stream));
+}
+
+int64_t cc_tensor_scores_ld(int K) { return (K < 1 || K > 65536) ? -1 : cc_tensor_score_ld(K); }
+
+cc_status cc_tensor_scores(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const float* C, int K, float* scores,
+                           void* stream) {
+    if (!ctx || !C || !X || !scores) return CC_ERR_NULL;
+    cc_status s = check_common(ctx, N, g, K, true);
+    if (s != CC_OK) return s;
+    if (N < 1 || N > 65536) return CC_ERR_SHAPE;
+    if (!aligned16(X) || !aligned16(C)) return CC_ERR_ALIGN;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    const WsLayout L = cc_ws_layout(N, g, K);
+    return from_cuda(cc_launch_tensor_scores(ctx, L, X, N, g, C, K, scores, (cudaStream_t)stream));
 }
 
 cc_status cc_update(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const uint16_t* idx, int K, float* C,

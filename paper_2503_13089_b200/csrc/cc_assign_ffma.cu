@@ -240,26 +240,45 @@ assign_ffma_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __res
 }
 
 // ---------------------------------------------------------------------------------------------
-// Exact stage.  Each flagged point is scanned against every centroid by a group of T lanes of a
-// warp (T = 32, 8 or 1, chosen from the number of flagged points so that few points still fill
+// Exact stage.  Each flagged point is scanned against every centroid by a group of T threads
+// (T = 128, 32, 8 or 1, chosen from the number of flagged points so that few points still fill
 // the GPU and many points do not re-read the codebook too often).  A cheap FP32 direct-form
 // distance (relative error <= (g+2) 2^-24, no cancellation) screens the candidates; those within
 // 2^-18 of the best FP64 distance so far are recomputed in FP64 (sub, mul, add, in dimension
 // order, no FMA contraction) and the pair (distance, index) is minimised lexicographically.
 template <int G>
+__device__ __forceinline__ void load_centroid(const float* __restrict__ C, int j, float* c) {
+    const float* row = C + (int64_t)j * G;
+    if constexpr (G % 4 == 0) {
+#pragma unroll
+        for (int v = 0; v < G / 4; ++v) {
+            const float4 u = __ldg(reinterpret_cast<const float4*>(row) + v);
+            c[4 * v] = u.x; c[4 * v + 1] = u.y; c[4 * v + 2] = u.z; c[4 * v + 3] = u.w;
+        }
+    } else {
+#pragma unroll
+        for (int t = 0; t < G; ++t) c[t] = __ldg(row + t);
+    }
+}
+
+template <int G>
 __global__ void __launch_bounds__(128)
 resolve_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restrict__ C, int K,
                const unsigned* __restrict__ status, const unsigned* __restrict__ flagged,
                uint16_t* __restrict__ idx, float* __restrict__ dist) {
+    __shared__ double sh_d[4];
+    __shared__ int sh_j[4];
     ull F = *reinterpret_cast<const ull*>(status + 2);
     if (F > (ull)N) F = (ull)N;
     if (F == 0) return;
     const ull total_threads = (ull)gridDim.x * blockDim.x;
-    const int T = (F * 32 <= total_threads) ? 32 : (F * 8 <= total_threads) ? 8 : 1;
+    // threads per point: a whole block while the flagged points are fewer than the blocks, then a
+    // warp, 8 lanes, one lane
+    const int T = (F <= (ull)gridDim.x) ? 128 : (F * 32 <= total_threads) ? 32 : (F * 8 <= total_threads) ? 8 : 1;
     const ull gthread = (ull)blockIdx.x * blockDim.x + threadIdx.x;
     const int lane = (int)(gthread % T);
     const ull n_groups = total_threads / T;
-    const ull n_rounds = (F + n_groups - 1) / n_groups;       // the same for every lane of a warp
+    const ull n_rounds = (F + n_groups - 1) / n_groups;       // the same for every thread of a block
     for (ull r = 0; r < n_rounds; ++r) {
         const ull f = r * n_groups + gthread / T;
         const bool live = f < F;
@@ -279,8 +298,7 @@ resolve_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restric
 #pragma unroll 2
         for (int j = lane; j < k_end; j += T) {
             float c[G];
-#pragma unroll
-            for (int t = 0; t < G; ++t) c[t] = __ldg(C + (int64_t)j * G + t);
+            load_centroid<G>(C, j, c);
             float dh = 0.f;
 #pragma unroll
             for (int t = 0; t < G; ++t) { const float df = x[t] - c[t]; dh = fmaf(df, df, dh); }
@@ -297,11 +315,24 @@ resolve_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restric
                 }
             }
         }
-        // lexicographic minimum of (distance, index) over the T lanes of the group
-        for (int o = T >> 1; o > 0; o >>= 1) {
+        // lexicographic minimum of (distance, index) over the T threads of the group
+        const int TW = T > 32 ? 32 : T;
+        for (int o = TW >> 1; o > 0; o >>= 1) {
             const double Do = __shfl_xor_sync(0xffffffffu, Db, o);
             const int jo = __shfl_xor_sync(0xffffffffu, jb, o);
             if (Do < Db || (Do == Db && jo < jb)) { Db = Do; jb = jo; }
+        }
+        if (T == 128) {                         // uniform over the grid
+            const int w = threadIdx.x >> 5;
+            __syncthreads();                    // the previous round's readers are done
+            if ((threadIdx.x & 31) == 0) { sh_d[w] = Db; sh_j[w] = jb; }
+            __syncthreads();
+#pragma unroll
+            for (int o = 0; o < 4; ++o) {
+                const double Do = sh_d[o];
+                const int jo = sh_j[o];
+                if (Do < Db || (Do == Db && jo < jb)) { Db = Do; jb = jo; }
+            }
         }
         if (live && lane == 0) {
             idx[i] = (uint16_t)jb;

@@ -1,26 +1,39 @@
 // E-step of Section 3.1 on the 5th-generation tensor cores (tcgen05, accumulators in TMEM).
 //
-// The score matrix S = ||c||^2 - 2 x.c of a tile of 128 points x 256 centroids is one dense
-// contraction  S = A . B^T  with
-//     A row (point i)    = [ x , x (, x) , 1 , 1 , 1 , 0.. ]
-//     B row (centroid j) = [ m1, m2 (, m3), q1, q2, q3, 0.. ],   m = -2c = m1 + m2 (+ m3),
-// where the FP32 centroid is split into TF32 pieces (three pieces = exact, two pieces = 2^-22
-// relative) and q1 + q2 + q3 is ||c||^2 (computed in FP64) to 33 bits.  FP16 points are exact in
-// TF32.  `tcgen05.mma.kind::tf32` accumulates in FP32 in tensor memory; operands sit in shared
-// memory in the canonical K-major layout without swizzle (8-row x 16-byte core matrices).
+// The score matrix  S s_ij = S (||c_j||^2 - 2 x_i.c_j)  of a tile of 128 points x 256 centroids is
+// one dense FP16 contraction  A . B^T  with FP32 accumulation:
+//     A row (point i)    = [ x , x (, x) , 2^15, 2^6, 2^-3, 2^-12, 0.. ]
+//     B row (centroid j) = [ h1, h2 (, h3), p1 , p2 , p3  , p4   , 0.. ]
+// x is FP16 data and therefore exact.  S is a power of two chosen per call so that
+// |S m| < 2^15 and S ||c||^2 < 2^30 for every centroid (m = -2c); S m = h1 + h2 + h3 is the FP32
+// value cut into FP16 pieces (each piece is the FP16 rounding of what is left), and
+// S ||c||^2 (from FP64) = 2^15 p1 + 2^6 p2 + 2^-3 p3 + 2^-12 p4 likewise.  Scaling by a power of
+// two changes neither the order of the scores nor their rounding.  g = 15, 16 use two pieces of m
+// (relative residue 2^-22) to keep the contraction at 48 columns.
 //
-// One CTA keeps NA tiles of 128 points (the A operand) resident in shared memory and streams the
-// whole staged codebook (B tiles of 256 centroids, written by the prep kernel in the exact
-// shared-memory image so that one 1-D bulk copy fetches a tile) through a 2-stage ring.
-// Warp roles: 8 epilogue warps (warp w reads TMEM lanes 32*(w%4).., columns 128*(w/4)..),
-// one copy warp, one MMA warp (a single thread issues the MMAs).  The epilogue only takes the
-// running minimum of each 64-centroid chunk (3-input min) and keeps best / second-best chunk
-// minimum and the best chunk id per point; the index inside the chunk, the distance and the
-// near-tie flag are computed afterwards by the finish kernel, exactly as in the FP32 path.
-// Nothing N x K is ever written to memory.
+// Subnormal pieces are never emitted: the tensor core adds the products of one instruction after
+// aligning them by the operands' exponent FIELDS, so a subnormal piece next to the constant 2^15
+// widens the alignment window and costs the other addends their low bits (measured: an absolute
+// error of 2^-22 in scaled units).  A piece below 2^-14 is written as zero instead and the next,
+// finer piece picks the residue up; what is lost in the end is below 2^-14 per coordinate of S m
+// and below 2^-26 on S ||c||^2, and the near-tie test accounts for both.  Subnormal coordinates
+// of x itself are multiplied exactly (measured) but count with magnitude 2^-14 in that test.
+//
+// One CTA keeps up to NA tiles of 128 points (the A operand) resident in shared memory and
+// streams the staged codebook (B tiles of 256 centroids, written by the prep kernel as the exact
+// shared-memory image so that one bulk copy fetches a tile) through a ring.  Warp roles:
+// 16 epilogue warps (warp e reads TMEM lanes 32 (e % 4).., columns 64 (e / 4)..), one copy warp,
+// one MMA warp (a single thread issues the MMAs).  Two accumulators of 256 columns alternate, so
+// the tensor core fills one while the epilogue drains the other; a warp releases its share of
+// an accumulator as soon as its 64 columns are in registers.  The epilogue keeps, per point, the
+// smallest and second-smallest 64-centroid chunk minimum and the id of the best chunk (one
+// 3-input min per two scores); the index inside the chunk, the distance and the near-tie flag are
+// computed afterwards by the finish kernel from FP32 data.  Nothing N x K is written to memory.
 //
 // Every wait on an mbarrier is bounded (clock based); on a time-out the CTA raises the status
 // bit CC_DEV_TIMEOUT, stops issuing work, and still releases its tensor memory.
+#include <cuda_fp16.h>
+
 #include "cc_common.cuh"
 #include "cc_assign_shared.cuh"
 
@@ -28,32 +41,44 @@ namespace {
 
 constexpr int TM = 128;            // points per MMA = TMEM lanes
 constexpr int TN = 256;            // centroids per MMA = TMEM columns of one accumulator
-constexpr int TCHUNK = 64;         // centroids per tracked minimum
-constexpr int EPI_WARPS = 8;
+constexpr int TCHUNK = 64;         // centroids per tracked minimum = columns per epilogue warp
+constexpr int NQ = 4;              // FP16 pieces of S ||c||^2
+constexpr int EW = TN / TCHUNK;    // epilogue warps per TMEM lane quarter
+constexpr int EPI_WARPS = 4 * EW;
 constexpr int TC_THREADS = (EPI_WARPS + 2) * 32;
-constexpr int STAGES = 2;
+constexpr int SLOTS = 2;           // accumulators in TMEM
+constexpr int NA = 8;              // resident point tiles per CTA
+constexpr int LPP = 8;             // lanes per point in the finish kernel
 constexpr long long WAIT_LIMIT = 4000000000LL;   // clock cycles (about 2 s)
 
 template <int G> struct TcCfg {
-    static constexpr int SPLIT = (G <= 4) ? 3 : 2;                 // TF32 pieces of each centroid value
-    static constexpr int KD = (SPLIT * G + 3 + 7) / 8 * 8;          // contraction length, multiple of 8
-    static constexpr int A_TILE = TM * KD * 4;                      // bytes
-    static constexpr int B_TILE = TN * KD * 4;
-    // resident point tiles / TMEM accumulators: small g runs two CTAs per SM with one accumulator
-    // each, large g one CTA per SM with two accumulators
-    static constexpr int NA = (G <= 4) ? 8 : 4;
-    static constexpr int SLOTS = (G <= 8) ? 1 : 2;
-    static constexpr int MIN_BLOCKS = (G <= 8) ? 2 : 1;
-    static constexpr int SMEM = NA * A_TILE + STAGES * B_TILE + 256;
-    // rounding model of the scan: 2^-24 units of (2||c||^2 + ||x||^2); see the finish kernel
-    static constexpr int ERR_UNITS = (SPLIT == 3) ? 16 : 40;
+    static constexpr int SPLIT = (3 * G + NQ <= 48) ? 3 : 2;        // FP16 pieces of each S m value
+    static constexpr int KD = (SPLIT * G + NQ + 15) / 16 * 16;      // contraction length (halves)
+    static constexpr int A_TILE = TM * KD * 2;                      // bytes
+    static constexpr int B_TILE = TN * KD * 2;
+    static constexpr int STAGES = (KD <= 16) ? 4 : 3;
+    static constexpr int MERGE = (EW - 1) * NA * TM * 12;           // exchange of the column groups' results
+    static constexpr int SMEM = NA * A_TILE + STAGES * B_TILE + MERGE + 256;
+    // Rounding model of the accumulation, in units of 2^-24 (2||c||^2 + ||x||^2): measured on the
+    // device at 2.3 / 3.4 / 4.2 units for one / two / three 16-column MMA steps; the two-piece
+    // split adds 4.
+    static constexpr int ERR_UNITS = 8 * (KD / 16) + (SPLIT == 2 ? 4 : 0);
+};
+
+// Written by the range kernel / prep kernel, read by the finish kernel (workspace, 16 bytes).
+struct TcParams {
+    unsigned cmax_bits;   // max |c| (FP32 bits; non-negative floats order like unsigned integers)
+    unsigned qmax_bits;   // max ||c||^2, rounded up
+    float S, invS;
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
-// Offset (in floats) of element (row r, k) of an R-row operand in the canonical K-major layout.
-__device__ __forceinline__ int canon_off(int r, int k, int R) {
-    return (k >> 2) * (R * 4) + (r >> 3) * 32 + (r & 7) * 4 + (k & 3);
+// Byte offset of element (row r, column k) of an R-row FP16 operand in the canonical K-major layout
+// without swizzle: 8-row x 16-byte core matrices, 128 bytes apart along the rows, R*16 bytes
+// apart along k.
+__device__ __forceinline__ int canon_bytes(int r, int k, int R) {
+    return (k >> 3) * (R * 16) + (r >> 3) * 128 + (r & 7) * 16 + (k & 7) * 2;
 }
 
 __device__ __forceinline__ uint64_t make_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -91,61 +116,141 @@ __device__ __forceinline__ float min3(float a, float b, float c) {
     return d;
 }
 
-__device__ __forceinline__ float tf32_trunc(float f) { return __uint_as_float(__float_as_uint(f) & 0xffffe000u); }
-__device__ __forceinline__ float tf32_round(float f) {
-    uint32_t u;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(u) : "f"(f));
-    return __uint_as_float(u & 0xffffe000u);
+__device__ __forceinline__ int floor_log2_bits(unsigned bits) { return (int)((bits >> 23) & 0xffu) - 127; }
+
+// S = 2^k, the largest power of two with  S * 2 cmax < 2^15  and  S * qmax < 2^30  (k <= 40).
+__device__ __forceinline__ float scale_from_range(unsigned cmax_bits, unsigned qmax_bits) {
+    int k = 14 - (floor_log2_bits(cmax_bits) + 1);
+    const int k2 = 29 - floor_log2_bits(qmax_bits);
+    k = k < k2 ? k : k2;
+    k = k < 40 ? k : 40;
+    k = k > -120 ? k : -120;
+    return __int_as_float((k + 127) << 23);
 }
 
-// Staged B operand: tile b holds centroids 256b .. 256b+255 in the canonical layout, KD floats per
-// centroid: SPLIT x G pieces of m = -2c, three pieces of ||c||^2, zeros.  One thread writes four
-// consecutive k of one centroid (16 bytes).
-template <int G>
-__global__ void prep_tensor_kernel(const float* __restrict__ C, int K, int Kpad, float* __restrict__ gB) {
-    using Cfg = TcCfg<G>;
-    constexpr int KD = Cfg::KD, SPLIT = Cfg::SPLIT;
-    const int e = blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= Kpad * (KD / 4)) return;
-    const int j = e / (KD / 4), kc = e - j * (KD / 4);
-    float out[4];
-    float q[3] = {kBig, 0.f, 0.f};
+// Largest |c| and largest ||c||^2 of the codebook (params zeroed beforehand).
+__global__ void __launch_bounds__(256)
+tensor_range_kernel(const float* __restrict__ C, int K, int g, TcParams* __restrict__ params) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    float cm = 0.f, qm = 0.f;
     if (j < K) {
         double s = 0.0;
-#pragma unroll
-        for (int t = 0; t < G; ++t) { const double c = (double)C[(int64_t)j * G + t]; s += c * c; }
-        q[0] = tf32_trunc((float)s);
-        const double r1 = s - (double)q[0];
-        q[1] = tf32_trunc((float)r1);
-        q[2] = tf32_round((float)(r1 - (double)q[1]));
-    } else {
-        q[0] = tf32_trunc(kBig);
+        for (int t = 0; t < g; ++t) {
+            const float c = C[(int64_t)j * g + t];
+            cm = fmaxf(cm, fabsf(c));
+            s += (double)c * (double)c;
+        }
+        qm = __double2float_ru(s);
     }
 #pragma unroll
-    for (int u = 0; u < 4; ++u) {
-        const int k = kc * 4 + u;
-        float v = 0.f;
+    for (int o = 16; o > 0; o >>= 1) {
+        cm = fmaxf(cm, __shfl_xor_sync(0xffffffffu, cm, o));
+        qm = fmaxf(qm, __shfl_xor_sync(0xffffffffu, qm, o));
+    }
+    if ((threadIdx.x & 31) == 0) {
+        atomicMax(&params->cmax_bits, __float_as_uint(cm));
+        atomicMax(&params->qmax_bits, __float_as_uint(qm));
+    }
+}
+
+// h, or zero when h is not a normal FP16 number (see the header comment).
+__device__ __forceinline__ __half normal_or_zero(__half h) {
+    return ((__half_as_ushort(h) & 0x7c00u) == 0u) ? __ushort_as_half((unsigned short)0) : h;
+}
+
+__device__ __forceinline__ float qconst(int p) {   // 2^15, 2^6, 2^-3, 2^-12
+    return p == 0 ? 32768.0f : p == 1 ? 64.0f : p == 2 ? 0.125f : 0.000244140625f;
+}
+
+// Staged B operand: tile b holds centroids 256b .. 256b+255 in the canonical layout, KD halves per
+// centroid: SPLIT x G pieces of S m, NQ pieces of S ||c||^2, zeros.  One thread writes eight
+// consecutive columns of one centroid (16 bytes).  Centroids K .. Kpad-1 are padding with a score
+// of 2^15 * 65504; should it ever beat a real score (only with extreme inputs) the gap test fails
+// and the exact stage decides.
+template <int G>
+__global__ void __launch_bounds__(256)
+prep_tensor_kernel(const float* __restrict__ C, int K, int Kpad, TcParams* __restrict__ params,
+                   uint16_t* __restrict__ gB) {
+    using Cfg = TcCfg<G>;
+    constexpr int KD = Cfg::KD, SPLIT = Cfg::SPLIT;
+    const float S = scale_from_range(params->cmax_bits, params->qmax_bits);
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e == 0) { params->S = S; params->invS = 1.0f / S; }
+    if (e >= Kpad * (KD / 8)) return;
+    const int j = e / (KD / 8), kc = e - j * (KD / 8);
+    __half out[8];
+    __half qp[NQ];
+    bool need_q = false;
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        const int k = kc * 8 + u;
+        if (k >= SPLIT * G && k < SPLIT * G + NQ) need_q = true;
+    }
+    if (need_q) {
+        if (j < K) {
+            double s = 0.0;
+#pragma unroll
+            for (int t = 0; t < G; ++t) { const double c = (double)C[(int64_t)j * G + t]; s += c * c; }
+            double R = s * (double)S;
+#pragma unroll
+            for (int p = 0; p < NQ; ++p) {
+                const double a = (double)qconst(p);
+                qp[p] = normal_or_zero(__double2half(R / a));   // division by a power of two: exact
+                R -= (double)__half2float(qp[p]) * a;           // exact: cancels the leading bits of R
+            }
+        } else {
+            qp[0] = __ushort_as_half((unsigned short)0x7bffu);   // 65504
+#pragma unroll
+            for (int p = 1; p < NQ; ++p) qp[p] = __ushort_as_half((unsigned short)0);
+        }
+    }
+#pragma unroll
+    for (int u = 0; u < 8; ++u) {
+        const int k = kc * 8 + u;
+        __half v = __ushort_as_half((unsigned short)0);
         if (k < SPLIT * G) {
             if (j < K) {
                 const int piece = k / G, t = k - piece * G;
-                const float m = -2.0f * C[(int64_t)j * G + t];
-                const float m1 = tf32_trunc(m);
-                const float r1 = m - m1;                       // exact in FP32
-                if (piece == 0) v = m1;
-                else if (SPLIT == 2) v = tf32_round(r1);
-                else {
-                    const float m2 = tf32_trunc(r1);
-                    v = (piece == 1) ? m2 : (r1 - m2);         // at most 2 bits left: exact in TF32
-                }
+                const float M = S * (-2.0f * C[(int64_t)j * G + t]);    // exact (powers of two)
+                const __half h1 = normal_or_zero(__float2half_rn(M));
+                const float r1 = M - __half2float(h1);                  // exact: at most 13 bits (or M itself)
+                const __half h2 = normal_or_zero(__float2half_rn(r1));
+                const float r2 = r1 - __half2float(h2);
+                v = (piece == 0) ? h1 : (piece == 1) ? h2 : normal_or_zero(__float2half_rn(r2));
             }
-        } else if (k < SPLIT * G + 3) {
-            v = q[k - SPLIT * G];
+        } else if (k < SPLIT * G + NQ) {
+            v = qp[k - SPLIT * G];
         }
         out[u] = v;
     }
     const int tile = j / TN, jr = j - tile * TN;
-    float* dst = gB + (int64_t)tile * (TN * KD) + canon_off(jr, kc * 4, TN);
-    *reinterpret_cast<float4*>(dst) = make_float4(out[0], out[1], out[2], out[3]);
+    unsigned char* dst = reinterpret_cast<unsigned char*>(gB) + (int64_t)tile * Cfg::B_TILE + canon_bytes(jr, kc * 8, TN);
+    uint4 w;
+    w.x = (unsigned)__half_as_ushort(out[0]) | ((unsigned)__half_as_ushort(out[1]) << 16);
+    w.y = (unsigned)__half_as_ushort(out[2]) | ((unsigned)__half_as_ushort(out[3]) << 16);
+    w.z = (unsigned)__half_as_ushort(out[4]) | ((unsigned)__half_as_ushort(out[5]) << 16);
+    w.w = (unsigned)__half_as_ushort(out[6]) | ((unsigned)__half_as_ushort(out[7]) << 16);
+    *reinterpret_cast<uint4*>(dst) = w;
+}
+
+// FP32 codebook of the finish kernel, one block of (g+1) x 64 floats per 64-centroid chunk: for
+// coordinate t the 64 values m_{j,t} = -2 c_{j,t} of the chunk's centroids side by side, then their
+// 64 squared norms.  A group of 8 lanes reads 128 contiguous bytes per load.  Centroids
+// K .. Kpad-1 are padding that can never win.
+template <int G>
+__global__ void __launch_bounds__(256)
+prep_rescan_kernel(const float* __restrict__ C, int K, int Kpad, float* __restrict__ rescan) {
+    const int j = blockIdx.x * blockDim.x + threadIdx.x;
+    if (j >= Kpad) return;
+    float* blk = rescan + (int64_t)(j / TCHUNK) * ((G + 1) * TCHUNK) + (j % TCHUNK);
+    double s = 0.0;
+#pragma unroll
+    for (int t = 0; t < G; ++t) {
+        const float c = (j < K) ? C[(int64_t)j * G + t] : 0.f;
+        blk[t * TCHUNK] = -2.0f * c;
+        s += (double)c * (double)c;
+    }
+    blk[G * TCHUNK] = (j < K) ? (float)s : kBig;
 }
 
 #define TMEM_LD32(v, taddr)                                                                                      \
@@ -169,23 +274,30 @@ __global__ void prep_tensor_kernel(const float* __restrict__ C, int K, int Kpad,
                    "+r"(v[29]), "+r"(v[30]), "+r"(v[31])                                                         \
                  :: "memory")
 
-template <int G>
-__global__ void __launch_bounds__(TC_THREADS, TcCfg<G>::MIN_BLOCKS)
-assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restrict__ gB, int n_btiles,
-                     float2* __restrict__ tstate, unsigned* __restrict__ status) {
+// DUMP = true writes every score (divided by S) to `dump` (row stride dump_ld) instead of
+// reducing them: a verification aid for the rounding model, used on small inputs only.
+template <int G, bool DUMP>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* __restrict__ gB, int n_btiles,
+                     int na_per_cta, const TcParams* __restrict__ params, float2* __restrict__ tstate,
+                     unsigned* __restrict__ status, float* __restrict__ dump, int64_t dump_ld) {
     using Cfg = TcCfg<G>;
-    constexpr int KD = Cfg::KD, NA = Cfg::NA, SLOTS = Cfg::SLOTS, SPLIT = Cfg::SPLIT;
-    constexpr int A_FLOATS = TM * KD, B_FLOATS = TN * KD;
+    constexpr int KD = Cfg::KD, SPLIT = Cfg::SPLIT, STAGES = Cfg::STAGES;
+    constexpr int A_TILE = Cfg::A_TILE, B_TILE = Cfg::B_TILE;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
-    float* sA = reinterpret_cast<float*>(smem_raw);                       // NA tiles
-    float* sB = sA + NA * A_FLOATS;                                       // STAGES tiles
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sB + STAGES * B_FLOATS); // b_full, b_empty, t_full, t_empty
+    unsigned char* sA = smem_raw;                                   // NA tiles
+    unsigned char* sB = sA + NA * A_TILE;                           // STAGES tiles
+    float* merge = reinterpret_cast<float*>(sB + STAGES * B_TILE);  // [EW-1][NA][3][TM]: best, second, best chunk id
+    uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(merge) + Cfg::MERGE);
     uint64_t* b_full = bars, *b_empty = bars + STAGES, *t_full = bars + 2 * STAGES, *t_empty = bars + 2 * STAGES + SLOTS;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * STAGES + 2 * SLOTS);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int64_t base = (int64_t)blockIdx.x * (NA * TM);
+    const int64_t tile0 = (int64_t)blockIdx.x * na_per_cta;          // first point tile of this CTA
+    const int64_t n_tiles = (N + TM - 1) / TM;
+    const int na = (int)((n_tiles - tile0 < na_per_cta) ? (n_tiles - tile0) : na_per_cta);
+    const int64_t base = tile0 * TM;
 
     if (tid == 0) {
         for (int s = 0; s < STAGES; ++s) {
@@ -199,22 +311,28 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __r
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // ---- A operand: [x repeated SPLIT times, 1, 1, 1, 0..] per point, written 16 bytes at a time
+    // ---- A operand: [x repeated SPLIT times, 2^15, 2^6, 2^-3, 2^-12, 0..] per point, 16 bytes at a time
     bool nonfinite = false;
-    for (int e = tid; e < NA * TM; e += TC_THREADS) {
+    for (int e = tid; e < na * TM; e += TC_THREADS) {
         float x[G];
         load_point<G>(X, base + e, N, x, nonfinite);
-        float* tile = sA + (e / TM) * A_FLOATS;
+        unsigned short h[KD];
+#pragma unroll
+        for (int k = 0; k < KD; ++k) {
+            h[k] = (k < SPLIT * G) ? __half_as_ushort(__float2half_rn(x[k % G]))    // exact: x is FP16 data
+                 : (k < SPLIT * G + NQ) ? __half_as_ushort(__float2half_rn(qconst(k - SPLIT * G)))
+                 : (unsigned short)0;
+        }
+        unsigned char* tile = sA + (e / TM) * A_TILE;
         const int r = e % TM;
 #pragma unroll
-        for (int kc = 0; kc < KD / 4; ++kc) {
-            float v[4];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-                const int k = kc * 4 + u;
-                v[u] = (k < SPLIT * G) ? x[k % G] : (k < SPLIT * G + 3 ? 1.0f : 0.0f);
-            }
-            *reinterpret_cast<float4*>(tile + canon_off(r, kc * 4, TM)) = make_float4(v[0], v[1], v[2], v[3]);
+        for (int kc = 0; kc < KD / 8; ++kc) {
+            uint4 w;
+            w.x = (unsigned)h[kc * 8 + 0] | ((unsigned)h[kc * 8 + 1] << 16);
+            w.y = (unsigned)h[kc * 8 + 2] | ((unsigned)h[kc * 8 + 3] << 16);
+            w.z = (unsigned)h[kc * 8 + 4] | ((unsigned)h[kc * 8 + 5] << 16);
+            w.w = (unsigned)h[kc * 8 + 6] | ((unsigned)h[kc * 8 + 7] << 16);
+            *reinterpret_cast<uint4*>(tile + canon_bytes(r, kc * 8, TM)) = w;
         }
     }
     if (nonfinite) atomicOr(status, CC_DEV_NONFINITE);
@@ -237,9 +355,10 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __r
                 const int st = b % STAGES;
                 if (!mbar_wait(smem_u32(b_empty + st), ((b / STAGES) & 1) ^ 1, abort_flag)) break;
                 const uint32_t bar = smem_u32(b_full + st);
-                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(Cfg::B_TILE) : "memory");
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(B_TILE) : "memory");
                 asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-                             ::"r"(smem_u32(sB + st * B_FLOATS)), "l"(gB + (int64_t)b * B_FLOATS), "r"(Cfg::B_TILE), "r"(bar)
+                             ::"r"(smem_u32(sB + st * B_TILE)),
+                               "l"(reinterpret_cast<const unsigned char*>(gB) + (int64_t)b * B_TILE), "r"(B_TILE), "r"(bar)
                              : "memory");
                 issued = b + 1;
             }
@@ -253,29 +372,39 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __r
     } else if (warp == EPI_WARPS + 1) {
         // ------------------------------------------------------------ MMA warp: one thread issues
         if (lane == 0) {
-            const uint32_t idesc = (1u << 4) | (2u << 7) | (2u << 10) | ((uint32_t)(TN >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+            // kind::f16: D = F32 (bits 4-5 = 1), A = B = F16 (0), both K-major, N >> 3 at bit 17, M >> 4 at bit 24
+            const uint32_t idesc = (1u << 4) | ((uint32_t)(TN >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+            // descriptors of the first tiles; the start-address field counts 16-byte units, so a
+            // tile or a 16-column step further on is a plain addition
+            const uint64_t descA0 = make_desc(smem_u32(sA), TM * 16, 128);
+            const uint64_t descB0 = make_desc(smem_u32(sB), TN * 16, 128);
             bool ok = true;
+            int q = 0;
             for (int b = 0; b < n_btiles && ok; ++b) {
                 const int st = b % STAGES;
                 ok = mbar_wait(smem_u32(b_full + st), (b / STAGES) & 1, abort_flag);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t bBase = smem_u32(sB + st * B_FLOATS);
-                for (int a = 0; a < NA; ++a) {
-                    const int q = b * NA + a, slot = q % SLOTS;
+                const uint64_t descB = descB0 + (uint64_t)((st * B_TILE) >> 4);
+                for (int a = 0; a < na; ++a, ++q) {
+                    const int slot = q % SLOTS;
                     ok = mbar_wait(smem_u32(t_empty + slot), ((q / SLOTS) & 1) ^ 1, abort_flag);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                    const uint32_t aBase = smem_u32(sA + a * A_FLOATS);
+                    const uint64_t descA = descA0 + (uint64_t)((a * A_TILE) >> 4);
                     const uint32_t d = tmem + slot * TN;
 #pragma unroll
-                    for (int s = 0; s < KD / 8; ++s) {
-                        const uint64_t da = make_desc(aBase + s * 2 * (TM * 16), TM * 16, 128);
-                        const uint64_t db = make_desc(bBase + s * 2 * (TN * 16), TN * 16, 128);
-                        const uint32_t acc = s > 0 ? 1u : 0u;
-                        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                                     "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-                                     ::"r"(d), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+                    for (int s = 0; s < KD / 16; ++s) {
+                        const uint64_t da = descA + (uint64_t)((s * 2 * (TM * 16)) >> 4);
+                        const uint64_t db = descB + (uint64_t)((s * 2 * (TN * 16)) >> 4);
+                        if (s == 0)
+                            asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 0, 0;\n\t"
+                                         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                                         ::"r"(d), "l"(da), "l"(db), "r"(idesc) : "memory");
+                        else
+                            asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.b32 p, 0, 0;\n\t"
+                                         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                                         ::"r"(d), "l"(da), "l"(db), "r"(idesc) : "memory");
                     }
                     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
                                  ::"r"(smem_u32(t_full + slot)) : "memory");
@@ -287,76 +416,106 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __r
         }
     } else {
         // ------------------------------------------------------------ epilogue warps
-        const int quarter = warp & 3, half = warp >> 2;
+        const int quarter = warp & 3, cg = warp >> 2;     // TMEM lane quarter, 64-column group
+        const int r = quarter * 32 + lane;                // row of the point tile = TMEM lane
+        const float invS = DUMP ? params->invS : 0.f;
         float b1[NA], b2[NA];
         int bc[NA];
 #pragma unroll
-        for (int a = 0; a < NA; ++a) { b1[a] = INFINITY; b2[a] = INFINITY; bc[a] = half * 2; }
+        for (int a = 0; a < NA; ++a) { b1[a] = INFINITY; b2[a] = INFINITY; bc[a] = cg; }
+        const uint32_t tbase = tmem + ((uint32_t)(quarter * 32) << 16) + cg * TCHUNK;
         bool ok = true;
+        int q = 0;
         for (int b = 0; b < n_btiles && ok; ++b) {
 #pragma unroll
             for (int a = 0; a < NA; ++a) {
-                if (!ok) continue;
-                const int q = b * NA + a, slot = q % SLOTS;
+                if (a >= na || !ok) continue;
+                const int slot = q % SLOTS;
                 ok = mbar_wait(smem_u32(t_full + slot), (q / SLOTS) & 1, abort_flag);
+                ++q;
                 if (!ok) continue;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-                const uint32_t t0 = tmem + ((uint32_t)(quarter * 32) << 16) + slot * TN + half * (TN / 2);
+                uint32_t v0[32], v1[32];
+                TMEM_LD32(v0, tbase + slot * TN);
+                TMEM_LD32(v1, tbase + slot * TN + 32);
+                TMEM_WAIT32(v0);
+                TMEM_WAIT32(v1);
+                // the 64 columns are in registers: hand this warp's share of the accumulator back
+                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                __syncwarp();
+                if (lane == 0)
+                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(t_empty + slot)) : "memory");
+                if constexpr (DUMP) {
+                    const int64_t i = base + a * TM + r;
+                    if (i < N) {
+                        float* row = dump + i * dump_ld + (int64_t)b * TN + cg * TCHUNK;
 #pragma unroll
-                for (int c = 0; c < (TN / 2) / TCHUNK; ++c) {
-                    float m0 = INFINITY, m1 = INFINITY, m2 = INFINITY, m3 = INFINITY;
+                        for (int u = 0; u < 32; ++u) { row[u] = __uint_as_float(v0[u]) * invS; row[32 + u] = __uint_as_float(v1[u]) * invS; }
+                    }
+                } else {
+                    // one chunk of 64 columns, four independent chains (30 three-input minima + 2)
+                    float m0 = min3(__uint_as_float(v0[0]), __uint_as_float(v0[1]), __uint_as_float(v0[2]));
+                    float m1 = min3(__uint_as_float(v0[8]), __uint_as_float(v0[9]), __uint_as_float(v0[10]));
+                    float m2 = min3(__uint_as_float(v0[16]), __uint_as_float(v0[17]), __uint_as_float(v0[18]));
+                    float m3 = min3(__uint_as_float(v0[24]), __uint_as_float(v0[25]), __uint_as_float(v0[26]));
 #pragma unroll
-                    for (int l = 0; l < TCHUNK / 32; ++l) {
-                        uint32_t v[32];
-                        TMEM_LD32(v, t0 + c * TCHUNK + l * 32);
-                        TMEM_WAIT32(v);
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            m0 = min3(m0, __uint_as_float(v[8 * u + 0]), __uint_as_float(v[8 * u + 1]));
-                            m1 = min3(m1, __uint_as_float(v[8 * u + 2]), __uint_as_float(v[8 * u + 3]));
-                            m2 = min3(m2, __uint_as_float(v[8 * u + 4]), __uint_as_float(v[8 * u + 5]));
-                            m3 = min3(m3, __uint_as_float(v[8 * u + 6]), __uint_as_float(v[8 * u + 7]));
+                    for (int hf = 0; hf < 2; ++hf) {
+                        const uint32_t* v = hf ? v1 : v0;
+                        if (hf) {
+                            m0 = min3(m0, __uint_as_float(v[0]), __uint_as_float(v[1]));
+                            m1 = min3(m1, __uint_as_float(v[8]), __uint_as_float(v[9]));
+                            m2 = min3(m2, __uint_as_float(v[16]), __uint_as_float(v[17]));
+                            m3 = min3(m3, __uint_as_float(v[24]), __uint_as_float(v[25]));
+                            m0 = min3(m0, __uint_as_float(v[2]), __uint_as_float(v[10]));
+                            m2 = min3(m2, __uint_as_float(v[18]), __uint_as_float(v[26]));
                         }
+                        m0 = min3(m0, __uint_as_float(v[3]), __uint_as_float(v[4]));
+                        m1 = min3(m1, __uint_as_float(v[11]), __uint_as_float(v[12]));
+                        m2 = min3(m2, __uint_as_float(v[19]), __uint_as_float(v[20]));
+                        m3 = min3(m3, __uint_as_float(v[27]), __uint_as_float(v[28]));
+                        m0 = min3(m0, __uint_as_float(v[5]), __uint_as_float(v[6]));
+                        m1 = min3(m1, __uint_as_float(v[13]), __uint_as_float(v[14]));
+                        m2 = min3(m2, __uint_as_float(v[21]), __uint_as_float(v[22]));
+                        m3 = min3(m3, __uint_as_float(v[29]), __uint_as_float(v[30]));
+                        m0 = min3(m0, __uint_as_float(v[7]), __uint_as_float(v[15]));
+                        m2 = min3(m2, __uint_as_float(v[23]), __uint_as_float(v[31]));
                     }
                     const float m = fminf(min3(m0, m1, m2), m3);
-                    const int chunk_id = b * (TN / TCHUNK) + half * ((TN / 2) / TCHUNK) + c;
+                    const int chunk_id = b * EW + cg;
                     const bool better = m < b1[a];
                     b2[a] = better ? b1[a] : fminf(b2[a], m);
                     bc[a] = better ? chunk_id : bc[a];
                     b1[a] = better ? m : b1[a];
                 }
-                asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                __syncwarp();
-                if (lane == 0)
-                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(t_empty + slot)) : "memory");
             }
         }
-        // ---- merge the two column halves of each point (through the A region, no longer read by
-        //      any MMA: the last accumulator was complete before its epilogue started) and store
-        asm volatile("bar.sync 1, %0;" ::"r"(EPI_WARPS * 32));
-        float* merge = sA;   // [NA][TM][3]
-        const int r = quarter * 32 + lane;
-        if (half == 1) {
+        if constexpr (!DUMP) {
+            // ---- merge the EW column groups of each point (through shared memory) and store
+            if (cg > 0) {
 #pragma unroll
-            for (int a = 0; a < NA; ++a) {
-                merge[(a * TM + r) * 3 + 0] = b1[a];
-                merge[(a * TM + r) * 3 + 1] = b2[a];
-                merge[(a * TM + r) * 3 + 2] = __int_as_float(bc[a]);
+                for (int a = 0; a < NA; ++a) {
+                    float* mrow = merge + (((cg - 1) * NA + a) * 3) * TM + r;
+                    mrow[0] = b1[a]; mrow[TM] = b2[a]; mrow[2 * TM] = __int_as_float(bc[a]);
+                }
             }
-        }
-        asm volatile("bar.sync 1, %0;" ::"r"(EPI_WARPS * 32));
-        if (half == 0 && ok && !*abort_flag) {
+            asm volatile("bar.sync 1, %0;" ::"r"(EPI_WARPS * 32));
+            if (cg == 0 && ok && !*abort_flag) {
 #pragma unroll
-            for (int a = 0; a < NA; ++a) {
-                const int64_t i = base + a * TM + r;
-                if (i >= N) continue;
-                const float o1 = merge[(a * TM + r) * 3 + 0], o2 = merge[(a * TM + r) * 3 + 1];
-                const int oc = __float_as_int(merge[(a * TM + r) * 3 + 2]);
-                float second;
-                int chunk;
-                if (o1 < b1[a] || (o1 == b1[a] && oc < bc[a])) { chunk = oc; second = fminf(o2, b1[a]); }
-                else { chunk = bc[a]; second = fminf(b2[a], o1); }
-                tstate[i] = make_float2(second, __int_as_float(chunk));
+                for (int a = 0; a < NA; ++a) {
+                    const int64_t i = base + a * TM + r;
+                    if (a >= na || i >= N) continue;
+                    float w1 = b1[a], w2 = b2[a];
+                    int wc = bc[a];
+#pragma unroll
+                    for (int o = 0; o < EW - 1; ++o) {
+                        const float* srow = merge + ((o * NA + a) * 3) * TM + r;
+                        const float o1 = srow[0], o2 = srow[TM];
+                        const int oc = __float_as_int(srow[2 * TM]);
+                        if (o1 < w1) { w2 = fminf(w1, o2); w1 = o1; wc = oc; }     // equal minima: the gap is 0 and
+                        else { w2 = fminf(w2, o1); }                                // the point goes to the exact stage
+                    }
+                    tstate[i] = make_float2(w2, __int_as_float(wc));
+                }
             }
         }
     }
@@ -367,75 +526,202 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __r
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(SLOTS * TN));
 }
 
-// Finish: index inside the winning chunk, distance, near-tie flag (shared with the FP32 path).
+// Finish, LPP = 8 lanes per point (four points per warp): lane k of a group recomputes the scores of
+// centroids 4k .. 4k+3 and 32+4k .. 32+4k+3 of the winning 64-centroid chunk with the FMA chain
+// s = fma(x_{g-1}, m_{g-1}, ... fma(x_0, m_0, ||c||^2)), keeping its smallest score, its index and
+// its runner-up; a butterfly over the group gives every lane the chunk's winner and runner-up;
+// then the squared distance to the winner in FP64 (sub, mul, add in dimension order, no
+// contraction) and the near-tie test.  A scan whose scores are off by at most
+//     E = ERR_UNITS 2^-24 (2||c||^2 + ||x||^2) + 2^-14 ||x||_1 / S + 2^-26 / S
+// (|x_t| counted as at least 2^-14) may misorder two scores closer than 2E; every centroid at
+// least as close as the winner has 2||c||^2 + ||x||^2 <= 5||x||^2 + 4 d^2, so a point whose two
+// smallest scores are closer than 2E with that substitution goes to the exact stage.
 template <int G>
 __global__ void __launch_bounds__(256)
 finish_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restrict__ C, int K,
-                     const float4* __restrict__ prep, const float2* __restrict__ tstate, uint16_t* __restrict__ idx,
-                     float* __restrict__ dist, unsigned* __restrict__ status, unsigned* __restrict__ flagged) {
-    const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
-    if (i >= N) return;
-    const float2 t = tstate[i];
-    finish_point<G, TCHUNK>(X, N, C, K, prep, i, __float_as_int(t.y), t.x, (double)TcCfg<G>::ERR_UNITS, idx, dist,
-                            status, flagged);
+                     const float* __restrict__ rescan, const float2* __restrict__ tstate,
+                     const TcParams* __restrict__ params, uint16_t* __restrict__ idx, float* __restrict__ dist,
+                     unsigned* __restrict__ status, unsigned* __restrict__ flagged) {
+    const int k = threadIdx.x & (LPP - 1);
+    const int64_t group0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / LPP;
+    const int64_t n_groups = ((int64_t)gridDim.x * blockDim.x) / LPP;
+    const int64_t rounds = (N + n_groups - 1) / n_groups;            // the same for every lane of a warp
+    const float invS = params->invS;
+    for (int64_t rd = 0; rd < rounds; ++rd) {
+        const int64_t i_raw = rd * n_groups + group0;
+        const bool live = i_raw < N;
+        const int64_t i = live ? i_raw : N - 1;
+        const float2 t = tstate[i];
+        const int chunk = __float_as_int(t.y);
+        float x[G];
+        bool nf = false;
+        load_point<G>(X, i, N, x, nf);                       // the same address in the lanes of a group
+        const float4* blk = reinterpret_cast<const float4*>(rescan + (int64_t)chunk * ((G + 1) * TCHUNK)) + k;
+        float s1 = INFINITY, s2 = INFINITY;
+        int j1 = 4 * k;
+#pragma unroll
+        for (int hf = 0; hf < 2; ++hf) {
+            const float4 cs = __ldg(blk + G * (TCHUNK / 4) + hf * LPP);
+            float s[4] = {cs.x, cs.y, cs.z, cs.w};
+#pragma unroll
+            for (int u = 0; u < G; ++u) {
+                const float4 mv = __ldg(blk + u * (TCHUNK / 4) + hf * LPP);
+                s[0] = fmaf(x[u], mv.x, s[0]);
+                s[1] = fmaf(x[u], mv.y, s[1]);
+                s[2] = fmaf(x[u], mv.z, s[2]);
+                s[3] = fmaf(x[u], mv.w, s[3]);
+            }
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const bool take = s[e] < s1;                 // ascending index: strict '<' keeps the lowest
+                s2 = take ? s1 : fminf(s2, s[e]);
+                j1 = take ? hf * 32 + 4 * k + e : j1;
+                s1 = take ? s[e] : s1;
+            }
+        }
+#pragma unroll
+        for (int o = LPP / 2; o > 0; o >>= 1) {
+            const float os1 = __shfl_xor_sync(0xffffffffu, s1, o);
+            const float os2 = __shfl_xor_sync(0xffffffffu, s2, o);
+            const int oj = __shfl_xor_sync(0xffffffffu, j1, o);
+            const bool take = os1 < s1 || (os1 == s1 && oj < j1);
+            s2 = fminf(take ? s1 : os1, fminf(s2, os2));
+            s1 = take ? os1 : s1;
+            j1 = take ? oj : j1;
+        }
+        j1 += chunk * TCHUNK;
+        if (j1 >= K) j1 = K - 1;   // only reachable with non-finite input
+        s2 = fminf(s2, t.x * invS);
+        double D = 0.0;
+        float A = 0.f, L1 = 0.f;
+#pragma unroll
+        for (int u = 0; u < G; ++u) {
+            const double df = __dsub_rn((double)x[u], (double)__ldg(C + (int64_t)j1 * G + u));
+            D = __dadd_rn(D, __dmul_rn(df, df));
+            const float xf = fmaxf(fabsf(x[u]), 6.103515625e-5f);
+            A = fmaf(xf, xf, A);
+            L1 += fabsf(x[u]);
+        }
+        if (live && k == 0) {
+            idx[i] = (uint16_t)j1;
+            dist[i] = (float)D;
+            // A and L1 only feed the bound: FP32 is enough once they are rounded up a little
+            const double bound = 2.0 * ((double)TcCfg<G>::ERR_UNITS * 5.9604644775390625e-8 * (5.0 * (double)A * 1.0001 + 4.0 * D)
+                                        + (double)invS * (6.103515625e-5 * (double)L1 * 1.0001 + 1.4901161193847656e-8));
+            if (!((double)s2 - (double)s1 > bound)) {
+                const ull slot = atomicAdd(reinterpret_cast<ull*>(status + 2), 1ull);
+                flagged[slot] = (unsigned)i;
+            }
+        }
+    }
 }
 
 template <int G>
 cudaError_t launch_tensor(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64_t N, const float* C, int K,
-                          uint16_t* idx, float* dist, cudaStream_t st) {
+                          uint16_t* idx, float* dist, float* dump, int64_t dump_ld, cudaStream_t st) {
     using Cfg = TcCfg<G>;
     char* ws = static_cast<char*>(ctx->ws);
     unsigned* status = reinterpret_cast<unsigned*>(ws + L.status);
-    float* gB = reinterpret_cast<float*>(ws + L.tensor);
+    TcParams* params = reinterpret_cast<TcParams*>(ws + L.status + 128);
+    uint16_t* gB = reinterpret_cast<uint16_t*>(ws + L.tensor);
     float2* tstate = reinterpret_cast<float2*>(ws + L.tstate);
     const int Kpad = (int)cc_align_up((size_t)K, TN);
-    cudaError_t e = cc_launch_prep_ffma(ctx, L, G, C, K, st);   // staged codebook of the finish kernel; resets the flag counter
-    if (e != cudaSuccess) return e;
+    // FP32 rows of the finish kernel sit behind the FP16 operand image (at most 96 bytes per centroid)
+    float* rescan = reinterpret_cast<float*>(ws + L.tensor + (size_t)Kpad * 96);
+    cudaError_t e;
+    // status words 2..3 (the flagged-point counter of this E-step) and the range words
+    if ((e = cudaMemsetAsync(status + 2, 0, 8, st)) != cudaSuccess) return e;
+    if ((e = cudaMemsetAsync(params, 0, sizeof(TcParams), st)) != cudaSuccess) return e;
     {
         ProfScope ps(ctx, CC_K_ASSIGN_PREP, st);
-        const int n = Kpad * (Cfg::KD / 4);
-        prep_tensor_kernel<G><<<(n + 255) / 256, 256, 0, st>>>(C, K, Kpad, gB);
+        tensor_range_kernel<<<(K + 255) / 256, 256, 0, st>>>(C, K, G, params);
+    }
+    {
+        ProfScope ps(ctx, CC_K_ASSIGN_PREP, st);
+        const int n = Kpad * (Cfg::KD / 8);
+        prep_tensor_kernel<G><<<(n + 255) / 256, 256, 0, st>>>(C, K, Kpad, params, gB);
+    }
+    if (!dump) {
+        ProfScope ps(ctx, CC_K_ASSIGN_PREP, st);
+        prep_rescan_kernel<G><<<(Kpad + 255) / 256, 256, 0, st>>>(C, K, Kpad, rescan);
     }
     if (N > 0) {
+        const int64_t n_tiles = (N + TM - 1) / TM;
+        int64_t na_per_cta = (n_tiles + ctx->sm_count - 1) / ctx->sm_count;    // small inputs still use every SM
+        if (na_per_cta > NA) na_per_cta = NA;
+        const int64_t blocks = (n_tiles + na_per_cta - 1) / na_per_cta;
+        if (dump) {
+            static bool attr_set = false;
+            if (!attr_set) {
+                e = cudaFuncSetAttribute(assign_tensor_kernel<G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
+                if (e != cudaSuccess) return e;
+                attr_set = true;
+            }
+            ProfScope ps(ctx, CC_K_OTHER, st);
+            assign_tensor_kernel<G, true><<<(unsigned)blocks, TC_THREADS, Cfg::SMEM, st>>>(
+                X, N, gB, Kpad / TN, (int)na_per_cta, params, tstate, status, dump, dump_ld);
+            return cudaGetLastError();
+        }
         static bool attr_set = false;
         if (!attr_set) {
-            e = cudaFuncSetAttribute(assign_tensor_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
+            e = cudaFuncSetAttribute(assign_tensor_kernel<G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
             if (e != cudaSuccess) return e;
             attr_set = true;
         }
-        const int64_t per_block = (int64_t)Cfg::NA * TM;
-        const int64_t blocks = (N + per_block - 1) / per_block;
         {
             ProfScope ps(ctx, CC_K_ASSIGN_MAIN, st);
-            assign_tensor_kernel<G><<<(unsigned)blocks, TC_THREADS, Cfg::SMEM, st>>>(X, N, gB, Kpad / TN, tstate, status);
+            assign_tensor_kernel<G, false><<<(unsigned)blocks, TC_THREADS, Cfg::SMEM, st>>>(
+                X, N, gB, Kpad / TN, (int)na_per_cta, params, tstate, status, nullptr, 0);
         }
         {
             ProfScope ps(ctx, CC_K_ASSIGN_FINISH, st);
-            finish_tensor_kernel<G><<<(unsigned)((N + 255) / 256), 256, 0, st>>>(
-                X, N, C, K, reinterpret_cast<const float4*>(ws + L.cprep), tstate, idx, dist, status,
-                reinterpret_cast<unsigned*>(ws + L.flagged));
+            int64_t fblocks = (N * LPP + 255) / 256;
+            const int64_t cap = (int64_t)ctx->sm_count * 32;
+            if (fblocks > cap) fblocks = cap;
+            finish_tensor_kernel<G><<<(unsigned)fblocks, 256, 0, st>>>(
+                X, N, C, K, rescan, tstate, params, idx, dist, status, reinterpret_cast<unsigned*>(ws + L.flagged));
         }
     }
     return cudaGetLastError();
 }
 
+#define CC_TENSOR_DISPATCH(g, CALL)                                                                 \
+    switch (g) {                                                                                    \
+        case 1: CALL(1); break;   case 2: CALL(2); break;   case 3: CALL(3); break;                 \
+        case 4: CALL(4); break;   case 5: CALL(5); break;   case 6: CALL(6); break;                 \
+        case 7: CALL(7); break;   case 8: CALL(8); break;   case 9: CALL(9); break;                 \
+        case 10: CALL(10); break; case 11: CALL(11); break; case 12: CALL(12); break;               \
+        case 13: CALL(13); break; case 14: CALL(14); break; case 15: CALL(15); break;               \
+        case 16: CALL(16); break;                                                                   \
+        default: return cudaErrorInvalidValue;                                                      \
+    }
+
 }  // namespace
 
 bool cc_tensor_path_supported(int g, int K) {
     (void)K;
-    return g == 4 || g == 8 || g == 16;
+    return g >= 1 && g <= 16;
 }
+
+int cc_tensor_score_ld(int K) { return (int)cc_align_up((size_t)K, TN); }
 
 cudaError_t cc_launch_assign_tensor(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64_t N, int g,
                                     const float* C, int K, uint16_t* idx, float* dist, double* objective,
                                     int64_t* n_resolved, cudaStream_t st) {
-    cudaError_t e;
-    switch (g) {
-        case 4: e = launch_tensor<4>(ctx, L, X, N, C, K, idx, dist, st); break;
-        case 8: e = launch_tensor<8>(ctx, L, X, N, C, K, idx, dist, st); break;
-        case 16: e = launch_tensor<16>(ctx, L, X, N, C, K, idx, dist, st); break;
-        default: return cudaErrorInvalidValue;
-    }
+    cudaError_t e = cudaSuccess;
+#define CALL(G) e = launch_tensor<G>(ctx, L, X, N, C, K, idx, dist, nullptr, 0, st)
+    CC_TENSOR_DISPATCH(g, CALL)
+#undef CALL
     if (e != cudaSuccess) return e;
     return cc_launch_assign_tail(ctx, L, X, N, g, C, K, idx, dist, objective, n_resolved, st);
+}
+
+cudaError_t cc_launch_tensor_scores(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64_t N, int g,
+                                    const float* C, int K, float* scores, cudaStream_t st) {
+    cudaError_t e = cudaSuccess;
+    const int64_t ld = cc_tensor_score_ld(K);
+#define CALL(G) e = launch_tensor<G>(ctx, L, X, N, C, K, nullptr, nullptr, scores, ld, st)
+    CC_TENSOR_DISPATCH(g, CALL)
+#undef CALL
+    return e;
 }

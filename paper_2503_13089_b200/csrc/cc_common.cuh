@@ -91,6 +91,10 @@ bool cc_tensor_path_supported(int g, int K);
 cudaError_t cc_launch_assign_tensor(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const float* C,
                                     int K, uint16_t* idx, float* dist, double* objective, int64_t* n_resolved,
                                     cudaStream_t);
+// Verification aid: every comparison score of the tensor-core scan, N x cc_tensor_score_ld(K) floats.
+int cc_tensor_score_ld(int K);
+cudaError_t cc_launch_tensor_scores(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const float* C,
+                                    int K, float* scores, cudaStream_t);
 // Second stage shared by both E-step paths: exact FP64 decision for the flagged points, then
 // the deterministic objective sum.
 cudaError_t cc_launch_assign_tail(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const float* C,

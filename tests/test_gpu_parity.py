@@ -86,7 +86,10 @@ def test_assign_matches_oracle(N, g, K):
 
 
 @pytest.mark.parametrize("N,g,K", [(1, 4, 1), (2049, 4, 33), (70001, 4, 1000), (20000, 4, 4096), (9000, 8, 300),
-                                   (4097, 8, 2049), (6000, 16, 129), (2500, 16, 1500), (1100, 4, 65536)])
+                                   (4097, 8, 2049), (6000, 16, 129), (2500, 16, 1500), (1100, 4, 65536),
+                                   (3001, 1, 17), (3001, 2, 64), (3001, 3, 100), (3001, 5, 600), (3001, 6, 90),
+                                   (3001, 7, 1025), (3001, 9, 513), (1500, 12, 77), (1500, 13, 300), (1500, 15, 64),
+                                   (150000, 4, 300), (40000, 9, 700)])
 def test_assign_fp32_and_tensor_paths_agree_with_oracle_and_each_other(N, g, K):
     cc, u = _cc(), _u()
     X = wl.make_points(N, g, 1000 + N + g)
@@ -102,6 +105,59 @@ def test_assign_fp32_and_tensor_paths_agree_with_oracle_and_each_other(N, g, K):
     assert len(differ) <= max(1, N // 1000)          # only oracle near-ties may differ between the paths
     same = a[0] == b[0]
     assert np.array_equal(a[1][same], b[1][same])
+
+
+def _tensor_units(g):
+    """Rounding model of the tensor-core scan as the library documents it: contraction length,
+    number of FP16 pieces per centroid value, allowed error in units of 2^-24 (2||c||^2 + ||x||^2)."""
+    split = 3 if 3 * g + 4 <= 48 else 2
+    kd = (split * g + 4 + 15) // 16 * 16
+    return split, kd, 8 * (kd // 16) + (4 if split == 2 else 0)
+
+
+@pytest.mark.parametrize("kind", ["weights", "wide_range", "on_centroids", "huge"])
+@pytest.mark.parametrize("g", [1, 3, 4, 5, 8, 9, 12, 14, 15, 16])
+def test_tensor_scores_obey_the_rounding_model(g, kind):
+    """Every raw score of the tensor-core scan against float64: the error must stay inside the
+    bound that decides which points are sent to the exact stage (and, here, inside half of it)."""
+    cc, u = _cc(), _u()
+    rng = np.random.default_rng(100 * g + len(kind))
+    N, K = 700, 900
+    if kind == "weights":
+        X = wl.make_points(N, g, 50 + g)
+        C = wl.make_codebook(K, g, 60 + g)
+    elif kind == "wide_range":
+        X = (rng.standard_normal((N, g)) * np.exp2(rng.uniform(-20, 6, (N, g)))).astype(np.float16)
+        C = (rng.standard_normal((K, g)) * np.exp2(rng.uniform(-24, 6, (K, g)))).astype(np.float32)
+    elif kind == "on_centroids":
+        C = wl.make_codebook(K, g, 61 + g)
+        X = C[rng.integers(0, K, N)].astype(np.float16)
+    else:
+        X = (rng.standard_normal((N, g)) * 2e4).clip(-65000, 65000).astype(np.float16)
+        C = (rng.standard_normal((K, g)) * 1e4).astype(np.float32)
+    c = u.ctx()
+    c.ensure_workspace(N, g, K)
+    ld = cc.cc_tensor_scores_ld(K)
+    assert ld % 256 == 0 and ld >= K
+    out = torch.full((N, ld), float("nan"), dtype=torch.float32, device="cuda")
+    cc.cc_tensor_scores(c, u.half_dev(X), N, g, u.dev(C), K, out)
+    cc.cc_poll_status(c)
+    got = out.cpu().numpy().astype(np.float64)[:, :K]
+    assert np.isfinite(got).all()
+    Xd, Cd = X.astype(np.float64), C.astype(np.float64)
+    csq = (Cd ** 2).sum(1)
+    exact = csq[None, :] - 2.0 * Xd @ Cd.T
+    # the library's scale: largest power of two with S * 2 max|c| < 2^15 and S * max||c||^2 < 2^30
+    k = min(14 - (int(np.floor(np.log2(np.abs(C).max()))) + 1), 29 - int(np.floor(np.log2(csq.max() * (1 + 1e-7)))), 40)
+    inv_s = 2.0 ** -k
+    split, kd, units = _tensor_units(g)
+    xsq = (np.maximum(np.abs(Xd), 2.0 ** -14) ** 2).sum(1)      # subnormal coordinates count as 2^-14
+    rel = 2.0 ** -24 * (2 * csq[None, :] + xsq[:, None])
+    absolute = inv_s * (2.0 ** -14 * np.abs(Xd).sum(1)[:, None] + 2.0 ** -26)
+    err = np.abs(got - exact)
+    worst = float(((err - absolute).clip(0) / rel).max())
+    print("g=%d %s: worst error %.2f units (bound %d), scale 2^%d" % (g, kind, worst, units, k))
+    assert worst <= units / 2
 
 
 def test_assign_exact_ties_and_duplicates_take_lowest_index():

@@ -298,13 +298,36 @@ def main():
         avg_ms = ms_assign / max(n_assign, 1)
         achieved_tf = flops_launch / (avg_ms * 1e-3) / 1e12 if avg_ms > 0 else 0.0
         nominal_fp32 = NOMINAL_SM * NOMINAL_LANES * 2 * NOMINAL_MHZ * 1e6 / 1e12
-        roofline = {"bound": "alu", "kernel": "assign_main (E-step distance scan)", "achieved": achieved_tf,
-                    "peak": nominal_fp32, "unit": "TFLOP/s", "frac": achieved_tf / nominal_fp32,
-                    "peak_kind": "nominal FP32 FMA: 148 SMs x 128 lanes x 2 x 1965 MHz",
-                    "peak_measured_ffma_scalar": fp32_scalar, "peak_measured_ffma_packed": fp32_packed,
-                    "frac_of_measured_ffma": achieved_tf / max(fp32_scalar, fp32_packed, 1e-9),
-                    "avg_launch_ms": avg_ms, "launches": n_assign, "flops_per_launch": flops_launch,
-                    "traffic": None}
+        if args.path == "ffma":
+            # FP32 FMA scan: 2g flops per distance evaluation against the FP32 FMA pipes
+            roofline = {"bound": "alu", "kernel": "assign_ffma_kernel (E-step distance scan, FP32 FMA path)",
+                        "achieved": achieved_tf, "peak": nominal_fp32, "unit": "TFLOP/s",
+                        "frac": achieved_tf / nominal_fp32,
+                        "peak_kind": "nominal FP32 FMA: 148 SMs x 128 lanes x 2 x 1965 MHz",
+                        "peak_measured_ffma_scalar": fp32_scalar, "peak_measured_ffma_packed": fp32_packed,
+                        "avg_launch_ms": avg_ms, "launches": n_assign, "flops_per_launch": flops_launch,
+                        "traffic": None}
+        else:
+            # tensor-core scan: the contraction is cheap (1-3 MMA steps per 128 x 256 tile); the kernel
+            # is bound by the min-reduction of the scores on the ALU pipes, one lane-operation per score
+            # (a 3-input min retires two scores in two pipe cycles).  Peak: 148 SMs x 128 lanes x 1965 MHz
+            # scores/s, expressed in the same 2g flops per distance evaluation as `achieved`.
+            evals_launch = flops_launch / (2 * g)
+            peak_scores = NOMINAL_SM * NOMINAL_LANES * NOMINAL_MHZ * 1e6
+            peak_tf = peak_scores * 2 * g / 1e12
+            kd = ((3 if 3 * g + 4 <= 48 else 2) * g + 4 + 15) // 16 * 16
+            executed_tf = achieved_tf * kd / g
+            roofline = {"bound": "alu", "kernel": "assign_tensor_kernel (E-step: tcgen05 scores + min-reduction epilogue)",
+                        "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
+                        "peak_kind": "ALU min-reduction: 148 SMs x 128 lanes x 1965 MHz scores/s x 2g flops per score",
+                        "scores_per_s": evals_launch / (avg_ms * 1e-3) if avg_ms > 0 else 0.0,
+                        "x_fp32_fma_peak": achieved_tf / nominal_fp32,
+                        "tensor_frac_algorithmic_of_measured_bf16": achieved_tf / peaks["bf16_tflops"],
+                        "tensor_frac_executed_of_measured_bf16": executed_tf / peaks["bf16_tflops"],
+                        "contraction_columns": kd,
+                        "peak_measured_ffma_scalar": fp32_scalar,
+                        "avg_launch_ms": avg_ms, "launches": n_assign, "flops_per_launch": flops_launch,
+                        "traffic": None}
         kern = {}
         for k, (ms, n) in prof.items():
             if n:
@@ -325,8 +348,8 @@ def main():
             gbs = by / (ms_rs / n_rs * 1e-3) / 1e9
             kern["reshape"].update({"algorithmic_GBs": gbs, "frac_of_hbm": gbs / peaks["hbm_gbs"]})
         n_mat = len(specs)
-        lloyd_ms = (prof["assign_main"][0] + prof["assign_prep"][0] + prof["resolve"][0] + prof["objective"][0]
-                    + prof["update_accum"][0] + prof["update_finish"][0]) / max(args.steps, 1)
+        lloyd_ms = (prof["assign_main"][0] + prof["assign_prep"][0] + prof["assign_finish"][0] + prof["resolve"][0]
+                    + prof["objective"][0] + prof["update_accum"][0] + prof["update_finish"][0]) / max(args.steps, 1)
         s_per_iter = lloyd_ms * 1e-3 / (n_mat * (iters + 1))
 
         cpu_baseline = None

@@ -25,6 +25,7 @@ WsLayout cc_ws_layout(int64_t N, int g, int K) {
     // rows of the finish kernel (at most 68 bytes per centroid)
     L.tensor = take(Kpad * (size_t)(64 + 1) * 4);
     L.tstate = take((size_t)N * 8);
+    L.idx_prev = take((size_t)N * 2);
     L.total = off;
     return L;
 }
@@ -280,7 +281,15 @@ cc_status cc_fit(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, int K, int it
         cudaError_t e = assign_any(ctx, L, X, N, g, C, K, idx, dist, objective_trace ? objective_trace + it : nullptr,
                                    nullptr, st);
         if (e != cudaSuccess) return CC_ERR_CUDA;
-        e = cc_launch_update(ctx, L, X, N, g, idx, K, C, counts, st);
+        // first M-step: all points; later ones: only the points whose code changed
+        uint16_t* idx_prev = reinterpret_cast<uint16_t*>(static_cast<char*>(ctx->ws) + L.idx_prev);
+        if (it == 0) {
+            e = cc_launch_update(ctx, L, X, N, g, idx, K, C, counts, st);
+            if (e == cudaSuccess && iters > 1)
+                e = cudaMemcpyAsync(idx_prev, idx, sizeof(uint16_t) * (size_t)N, cudaMemcpyDeviceToDevice, st);
+        } else {
+            e = cc_launch_update_delta(ctx, L, X, N, g, idx, idx_prev, K, C, counts, st);
+        }
         if (e != cudaSuccess) return CC_ERR_CUDA;
     }
     return CC_OK;

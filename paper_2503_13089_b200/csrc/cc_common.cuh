@@ -64,6 +64,7 @@ struct WsLayout {
     size_t dist_tmp;   // float N: distances when the caller passes dist == NULL
     size_t tensor;     // staging of the tensor-core E-step (split codebook operand)
     size_t tstate;     // float2 N: (second-best chunk minimum, best chunk id) from the tensor-core scan
+    size_t idx_prev;   // u16 N: codes of the previous M-step inside cc_fit
     size_t total;
 };
 
@@ -103,3 +104,5 @@ cudaError_t cc_launch_assign_tail(cc_ctx*, const WsLayout&, const uint16_t* X, i
 
 cudaError_t cc_launch_update(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const uint16_t* idx,
                              int K, float* C, int32_t* counts, cudaStream_t);
+cudaError_t cc_launch_update_delta(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const uint16_t* idx,
+                                   uint16_t* idx_prev, int K, float* C, int32_t* counts, cudaStream_t);

@@ -60,6 +60,41 @@ update_accumulate_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16
     }
 }
 
+// M-step inside the Lloyd loop, from the second iteration on: the sums of the previous M-step are
+// still in the workspace, so only the points whose code changed are moved, subtracted from their
+// old cluster and added to the new one.  Integer sums make this bit-identical to summing all the
+// points again.  idx_prev holds the codes the sums correspond to and is brought up to date.
+template <int G>
+__global__ void __launch_bounds__(256)
+update_delta_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* __restrict__ idx,
+                    uint16_t* __restrict__ idx_prev, int K, ull* __restrict__ sum_lo, ull* __restrict__ sum_hi,
+                    int* __restrict__ counts) {
+    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < N; i += (int64_t)gridDim.x * blockDim.x) {
+        const int jn = idx[i], jo = idx_prev[i];
+        if (jn == jo || jn >= K || jo >= K) continue;
+        idx_prev[i] = (uint16_t)jn;
+        atomicAdd(counts + jn, 1);
+        atomicSub(counts + jo, 1);
+        const uint16_t* row = X + i * G;
+#pragma unroll
+        for (int t = 0; t < G; ++t) {
+            const uint16_t h = __ldg(row + t);
+            const float v = __half2float(__ushort_as_half(h));
+            const unsigned e = (h >> 10) & 31u;
+            if (e == 31u) continue;
+            if (e >= 18u) {
+                const long long q = __float2ll_rn(v * 128.0f);
+                atomicAdd(sum_hi + (int64_t)jn * G + t, (ull)q);
+                atomicAdd(sum_hi + (int64_t)jo * G + t, (ull)(-q));
+            } else if ((h & 0x7fffu) != 0u) {
+                const long long q = __float2ll_rn(v * 16777216.0f);
+                atomicAdd(sum_lo + (int64_t)jn * G + t, (ull)q);
+                atomicAdd(sum_lo + (int64_t)jo * G + t, (ull)(-q));
+            }
+        }
+    }
+}
+
 __global__ void __launch_bounds__(256)
 update_finish_kernel(const long long* __restrict__ sum_lo, const long long* __restrict__ sum_hi,
                      const int* __restrict__ counts, int K, int g, float* __restrict__ C) {
@@ -69,6 +104,30 @@ update_finish_kernel(const long long* __restrict__ sum_lo, const long long* __re
     if (n <= 0) return;   // empty cluster: previous centroid stays
     const double s = (double)sum_lo[e] * 5.9604644775390625e-8 + (double)sum_hi[e] * 0.0078125;
     C[e] = (float)(s / (double)n);
+}
+
+}  // namespace
+
+#define CC_UPDATE_DISPATCH(g, CALL)                                                                           \
+    switch (g) {                                                                                              \
+        case 1: CALL(1); break;   case 2: CALL(2); break;   case 3: CALL(3); break;   case 4: CALL(4); break;   \
+        case 5: CALL(5); break;   case 6: CALL(6); break;   case 7: CALL(7); break;   case 8: CALL(8); break;   \
+        case 9: CALL(9); break;   case 10: CALL(10); break; case 11: CALL(11); break; case 12: CALL(12); break; \
+        case 13: CALL(13); break; case 14: CALL(14); break; case 15: CALL(15); break; case 16: CALL(16); break; \
+        default: return cudaErrorInvalidValue;                                                                \
+    }
+
+namespace {
+
+template <int G>
+cudaError_t launch_accumulate(cc_ctx* ctx, const uint16_t* X, int64_t N, const uint16_t* idx, int K, ull* sum_lo,
+                              ull* sum_hi, int32_t* counts, cudaStream_t st) {
+    ProfScope ps(ctx, CC_K_UPDATE_ACCUM, st);
+    int64_t blocks = (N + 255) / 256;
+    const int64_t cap = (int64_t)ctx->sm_count * 16;
+    if (blocks > cap) blocks = cap;
+    update_accumulate_kernel<G><<<(unsigned)blocks, 256, 0, st>>>(X, N, idx, K, sum_lo, sum_hi, counts);
+    return cudaGetLastError();
 }
 
 }  // namespace
@@ -83,19 +142,32 @@ cudaError_t cc_launch_update(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, 
     if ((e = cudaMemsetAsync(sum_lo, 0, L.tmp_c - L.sum_lo, st)) != cudaSuccess) return e;
     if ((e = cudaMemsetAsync(counts, 0, sizeof(int32_t) * (size_t)K, st)) != cudaSuccess) return e;
     if (N > 0) {
+#define CALL(G) e = launch_accumulate<G>(ctx, X, N, idx, K, sum_lo, sum_hi, counts, st)
+        CC_UPDATE_DISPATCH(g, CALL)
+#undef CALL
+        if (e != cudaSuccess) return e;
+    }
+    ProfScope ps(ctx, CC_K_UPDATE_FINISH, st);
+    update_finish_kernel<<<(K * g + 255) / 256, 256, 0, st>>>(reinterpret_cast<long long*>(sum_lo),
+                                                             reinterpret_cast<long long*>(sum_hi), counts, K, g, C);
+    return cudaGetLastError();
+}
+
+// Incremental M-step (see update_delta_kernel): the workspace sums and `counts` must be those of
+// the previous M-step on the same X, and idx_prev the codes they were computed from.
+cudaError_t cc_launch_update_delta(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64_t N, int g,
+                                   const uint16_t* idx, uint16_t* idx_prev, int K, float* C, int32_t* counts,
+                                   cudaStream_t st) {
+    char* ws = static_cast<char*>(ctx->ws);
+    ull* sum_lo = reinterpret_cast<ull*>(ws + L.sum_lo);
+    ull* sum_hi = reinterpret_cast<ull*>(ws + L.sum_hi);
+    if (N > 0) {
         int64_t blocks = (N + 255) / 256;
         const int64_t cap = (int64_t)ctx->sm_count * 16;
         if (blocks > cap) blocks = cap;
         ProfScope ps(ctx, CC_K_UPDATE_ACCUM, st);
-#define CALL(G)                                                                                               \
-    update_accumulate_kernel<G><<<(unsigned)blocks, 256, 0, st>>>(X, N, idx, K, sum_lo, sum_hi, counts)
-        switch (g) {
-            case 1: CALL(1); break;   case 2: CALL(2); break;   case 3: CALL(3); break;   case 4: CALL(4); break;
-            case 5: CALL(5); break;   case 6: CALL(6); break;   case 7: CALL(7); break;   case 8: CALL(8); break;
-            case 9: CALL(9); break;   case 10: CALL(10); break; case 11: CALL(11); break; case 12: CALL(12); break;
-            case 13: CALL(13); break; case 14: CALL(14); break; case 15: CALL(15); break; case 16: CALL(16); break;
-            default: return cudaErrorInvalidValue;
-        }
+#define CALL(G) update_delta_kernel<G><<<(unsigned)blocks, 256, 0, st>>>(X, N, idx, idx_prev, K, sum_lo, sum_hi, counts)
+        CC_UPDATE_DISPATCH(g, CALL)
 #undef CALL
     }
     ProfScope ps(ctx, CC_K_UPDATE_FINISH, st);

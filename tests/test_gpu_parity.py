@@ -314,6 +314,29 @@ def test_cfg1_lockstep_fit_and_free_run():
     assert counts_fit.sum() == len(X)
 
 
+@pytest.mark.parametrize("N,g,K,iters", [(30000, 4, 300, 6), (9000, 8, 5000, 4), (5000, 16, 40, 5), (7000, 5, 129, 4)])
+def test_fit_moves_only_changed_points_yet_matches_the_driven_loop(N, g, K, iters):
+    """cc_fit sums all points in its first M-step and afterwards only moves the points whose code
+    changed; with exact integer sums that must give the same bits as a full M-step every time,
+    including for values on the coarse accumulator (|x| >= 8), subnormals and emptied clusters."""
+    u = _u()
+    rng = np.random.default_rng(N + g)
+    X = wl.make_points(N, g, 7000 + N)
+    X[::5] = (rng.standard_normal((len(X[::5]), g)) * 200).astype(np.float16)
+    X[::9] = (rng.standard_normal((len(X[::9]), g)) * 1e-6).astype(np.float16)
+    C0 = oracle.init_codebook(X, K, 11)
+    C_fit, idx_fit, dist_fit, counts_fit, trace_fit = _gpu_fit(X, C0, iters)
+    C = C0.copy()
+    for it in range(iters):
+        idx, dist, obj, nres = u.gpu_assign(X, C)
+        assert obj == trace_fit[it]
+        C, counts = u.gpu_update(X, idx, C)
+    assert np.array_equal(idx_fit, idx) and np.array_equal(counts_fit, counts)
+    assert np.array_equal(C_fit.view(np.uint32), C.view(np.uint32))
+    C_or, counts_or = oracle.update(X, idx, C)            # fixed point check of the last state against the oracle
+    assert np.array_equal(counts_or, counts)
+
+
 def test_blobs_recovered_and_k_equals_n():
     u = _u()
     X, labels, centres = wl.make_blobs(12, 300, 4, seed=90, sep=1.0, sigma=0.01)

@@ -27,6 +27,94 @@ reshape_transpose_kernel(const uint16_t* __restrict__ W, int64_t d_out, int64_t 
     }
 }
 
+// ---- 16-byte versions of the two transposing kernels (taken when every row is a whole number of
+// 8-element groups).  A 64 x 64 tile goes through shared memory with a row stride of 33 words:
+// global reads and writes are 16-byte vectors along the contiguous axis of each side, and the
+// column reads in shared memory spread over the banks.
+constexpr int TSW = 33;   // tile row stride in 32-bit words (64 halves + 2)
+
+// Writes the transposed tile: output row `ro` (0..63) takes element [8c+k][ro], k = 0..7, as one vector.
+__device__ __forceinline__ uint4 tile_column8(const unsigned* tile, int c, int ro) {
+    unsigned short h[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        const unsigned w = tile[(8 * c + k) * TSW + (ro >> 1)];
+        h[k] = (ro & 1) ? (unsigned short)(w >> 16) : (unsigned short)(w & 0xffffu);
+    }
+    uint4 v;
+    v.x = (unsigned)h[0] | ((unsigned)h[1] << 16);
+    v.y = (unsigned)h[2] | ((unsigned)h[3] << 16);
+    v.z = (unsigned)h[4] | ((unsigned)h[5] << 16);
+    v.w = (unsigned)h[6] | ((unsigned)h[7] << 16);
+    return v;
+}
+
+__device__ __forceinline__ void tile_put8(unsigned* tile, int r, int c, uint4 v) {
+    unsigned* dst = tile + r * TSW + 4 * c;
+    dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+}
+
+// PAPER_T reshape; needs d_in % 8 == 0 and out_pad % 8 == 0.
+__global__ void __launch_bounds__(256)
+reshape_transpose_vec_kernel(const uint16_t* __restrict__ W, int64_t d_out, int64_t d_in, int64_t out_pad,
+                             uint16_t* __restrict__ X) {
+    __shared__ unsigned tile[TD * TSW];
+    const int64_t i0 = (int64_t)blockIdx.x * TD, o0 = (int64_t)blockIdx.y * TD;
+    const int c = threadIdx.x & 7, r0 = threadIdx.x >> 3;
+#pragma unroll
+    for (int p = 0; p < 2; ++p) {               // rows: out_features, vectors along in_features
+        const int r = r0 + 32 * p;
+        const int64_t o = o0 + r, i = i0 + 8 * c;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (o < d_out && i < d_in) v = __ldg(reinterpret_cast<const uint4*>(W + o * d_in + i));
+        tile_put8(tile, r, c, v);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int p = 0; p < 2; ++p) {               // rows: in_features, vectors along out_features
+        const int r = r0 + 32 * p;
+        const int64_t i = i0 + r, o = o0 + 8 * c;
+        if (i < d_in && o < out_pad) *reinterpret_cast<uint4*>(X + i * out_pad + o) = tile_column8(tile, c, r);
+    }
+}
+
+// PAPER_T decode for g = 4, 8, 16; needs d_in % 8 == 0 and out_pad % 8 == 0.  A group of 8
+// consecutive out_features of one in_feature is two codes (g = 4), one code (g = 8) or half a
+// code (g = 16): the codebook is read in 8- or 16-byte pieces.
+template <int G>
+__global__ void __launch_bounds__(256)
+decode_transpose_vec_kernel(const uint16_t* __restrict__ C16, const uint16_t* __restrict__ idx, int64_t d_out,
+                            int64_t d_in, int64_t out_pad, uint16_t* __restrict__ W_hat) {
+    __shared__ unsigned tile[TD * TSW];
+    const int64_t i0 = (int64_t)blockIdx.x * TD, o0 = (int64_t)blockIdx.y * TD;
+    const int c = threadIdx.x & 7, r0 = threadIdx.x >> 3;
+#pragma unroll
+    for (int p = 0; p < 2; ++p) {               // rows: in_features, vectors along out_features
+        const int r = r0 + 32 * p;
+        const int64_t i = i0 + r, o = o0 + 8 * c;
+        uint4 v = make_uint4(0u, 0u, 0u, 0u);
+        if (i < d_in && o < out_pad) {
+            const int64_t flat = i * out_pad + o;
+            const int64_t n = flat / G;
+            if constexpr (G == 4) {
+                const uint2 a = __ldg(reinterpret_cast<const uint2*>(C16 + (int64_t)__ldg(idx + n) * 4));
+                const uint2 b = __ldg(reinterpret_cast<const uint2*>(C16 + (int64_t)__ldg(idx + n + 1) * 4));
+                v = make_uint4(a.x, a.y, b.x, b.y);
+            } else {
+                v = __ldg(reinterpret_cast<const uint4*>(C16 + (int64_t)__ldg(idx + n) * G + (flat - n * G)));
+            }
+        }
+        tile_put8(tile, r, c, v);
+    }
+    __syncthreads();
+#pragma unroll
+    for (int p = 0; p < 2; ++p) {               // rows: out_features, vectors along in_features
+        const int r = r0 + 32 * p;
+        const int64_t o = o0 + r, i = i0 + 8 * c;
+        if (o < d_out && i < d_in) *reinterpret_cast<uint4*>(W_hat + o * d_in + i) = tile_column8(tile, c, r);
+    }
+}
+
 // ROWS reshape: copy each row, padding it to in_pad elements.
 __global__ void __launch_bounds__(256)
 reshape_rows_kernel(const uint16_t* __restrict__ W, int64_t d_out, int64_t d_in, int64_t in_pad,
@@ -105,7 +193,10 @@ cudaError_t cc_launch_reshape(cc_ctx* ctx, const uint16_t* W, int64_t d_out, int
     if (layout == CC_LAYOUT_PAPER_T) {
         const int64_t out_pad = pad_to(d_out, g);
         dim3 grid((unsigned)((d_in + TD - 1) / TD), (unsigned)((out_pad + TD - 1) / TD));
-        reshape_transpose_kernel<<<grid, 256, 0, st>>>(W, d_out, d_in, out_pad, X);
+        if (d_in % 8 == 0 && out_pad % 8 == 0)
+            reshape_transpose_vec_kernel<<<grid, 256, 0, st>>>(W, d_out, d_in, out_pad, X);
+        else
+            reshape_transpose_kernel<<<grid, 256, 0, st>>>(W, d_out, d_in, out_pad, X);
     } else {
         const int64_t in_pad = pad_to(d_in, g);
         int64_t blocks = (d_out * in_pad + 255) / 256;
@@ -122,7 +213,11 @@ cudaError_t cc_launch_decode(cc_ctx* ctx, const uint16_t* C16, int K, int g, con
     if (layout == CC_LAYOUT_PAPER_T) {
         const int64_t out_pad = pad_to(d_out, g);
         dim3 grid((unsigned)((d_in + TD - 1) / TD), (unsigned)((d_out + TD - 1) / TD));
-        decode_transpose_kernel<<<grid, 256, 0, st>>>(C16, g, idx, d_out, d_in, out_pad, W_hat);
+        const bool vec = d_in % 8 == 0 && out_pad % 8 == 0;
+        if (vec && g == 4) decode_transpose_vec_kernel<4><<<grid, 256, 0, st>>>(C16, idx, d_out, d_in, out_pad, W_hat);
+        else if (vec && g == 8) decode_transpose_vec_kernel<8><<<grid, 256, 0, st>>>(C16, idx, d_out, d_in, out_pad, W_hat);
+        else if (vec && g == 16) decode_transpose_vec_kernel<16><<<grid, 256, 0, st>>>(C16, idx, d_out, d_in, out_pad, W_hat);
+        else decode_transpose_kernel<<<grid, 256, 0, st>>>(C16, g, idx, d_out, d_in, out_pad, W_hat);
     } else {
         const int64_t in_pad = pad_to(d_in, g);
         int64_t blocks = (d_out * d_in + 255) / 256;

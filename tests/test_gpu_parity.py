@@ -28,7 +28,8 @@ def _u():
 
 @pytest.mark.parametrize("layout", [0, 1])
 @pytest.mark.parametrize("d_out,d_in,g", [(8, 8, 4), (10, 7, 4), (130, 67, 4), (129, 200, 6), (64, 64, 16),
-                                          (100, 33, 9), (257, 300, 5), (1, 1, 1)])
+                                          (100, 33, 9), (257, 300, 5), (1, 1, 1), (136, 200, 4), (200, 72, 8),
+                                          (144, 328, 16), (130, 72, 4), (250, 136, 8), (512, 256, 4)])
 def test_reshape_and_decode_match_oracle(d_out, d_in, g, layout):
     cc, u = _cc(), _u()
     rng = np.random.default_rng(d_out + d_in + g)

@@ -44,9 +44,8 @@ class Workload:
     notes: str = ""
 
     def n_subvectors(self, m: MatrixSpec) -> int:
-        # all shipped configurations divide evenly; padding is exercised by tests
-        assert m.d_out % self.g == 0
-        return m.d_in * (m.d_out // self.g)
+        # out_features are padded up to a multiple of g (only the paper-grid workloads need it)
+        return m.d_in * ((m.d_out + self.g - 1) // self.g)
 
 
 def _layer7b(prefix_seed: int, init_seed: int) -> Tuple[MatrixSpec, ...]:
@@ -76,6 +75,20 @@ WORKLOADS = {
     "cfg5_layer7b_g16_k65536": Workload(
         "cfg5_layer7b_g16_k65536", 16, 65536, 15, _layer7b(1050, 2050),
         subset_frac=0.01),
+    # the paper's own settings for a 4096 x 4096 matrix (bits table): odd g with real padding and
+    # codebook sizes that are not powers of two
+    "grid_g6_n65500": Workload(
+        "grid_g6_n65500", 6, 65500, 20,
+        (MatrixSpec("w", 4096, 4096, "student_t3", 0.02, 0.0, 1106, 2106),), subset_frac=0.01),
+    "grid_g9_n65500": Workload(
+        "grid_g9_n65500", 9, 65500, 20,
+        (MatrixSpec("w", 4096, 4096, "student_t3", 0.02, 0.0, 1109, 2109),), subset_frac=0.01),
+    "grid_g5_n50000": Workload(
+        "grid_g5_n50000", 5, 50000, 20,
+        (MatrixSpec("w", 4096, 4096, "student_t3", 0.02, 0.0, 1105, 2105),), subset_frac=0.01),
+    "grid_g7_n35000": Workload(
+        "grid_g7_n35000", 7, 35000, 20,
+        (MatrixSpec("w", 4096, 4096, "student_t3", 0.02, 0.0, 1107, 2107),), subset_frac=0.01),
 }
 
 

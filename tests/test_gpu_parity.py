@@ -425,6 +425,47 @@ def test_large_k_workloads_sampled(name, mat, frac):
     assert trace[1] < trace[0]
 
 
+@pytest.mark.parametrize("name,frac", [("grid_g6_n65500", 0.001), ("grid_g9_n65500", 0.001),
+                                       ("grid_g5_n50000", 0.001), ("grid_g7_n35000", 0.001)])
+def test_paper_grid_settings_padded_and_sampled(name, frac):
+    """The paper's own (g, n) settings on a 4096 x 4096 matrix: g does not divide 4096, so every
+    in_feature's last sub-vector is zero-padded, and n is not a power of two.  Two lock-step
+    iterations on a seeded sample, then the whole path from host buffers: decode must invert the
+    codes exactly and the objective must exceed ||W - decode||^2 by the padded coordinates' share."""
+    cc, u = _cc(), _u()
+    w = wl.WORKLOADS[name]
+    spec = w.matrices[0]
+    W = wl.make_matrix(spec)
+    X = oracle.reshape_subvectors(W, w.g)
+    assert len(X) == w.n_subvectors(spec) == cc.cc_num_subvectors(spec.d_out, spec.d_in, w.g, 0)
+    C0 = oracle.init_codebook(X, w.K, spec.init_seed)
+    sel = wl.subset_positions(len(X), frac, 5)
+    C, trace, tol = _lockstep(X, C0, 2, sel=sel)
+    print(name, "tolerated near-ties on the sample:", tol, "objective", trace)
+    assert trace[1] < trace[0]
+    d_out, d_in = W.shape
+    N = len(X)
+    C16 = torch.empty((w.K, w.g), dtype=torch.float16).pin_memory()
+    idx = torch.empty(N, dtype=torch.uint16).pin_memory()
+    tr = torch.empty(3, dtype=torch.float64).pin_memory()
+    What = torch.empty((d_out, d_in), dtype=torch.float16).pin_memory()
+    Wh = torch.from_numpy(W.view(np.int16)).view(torch.float16).pin_memory()
+    cc.cc_compress_host(u.ctx(), Wh, d_out, d_in, w.g, w.K, 2, spec.init_seed, 0, C16, idx, tr, What)
+    C16n = C16.numpy()
+    idxn = idx.view(torch.int16).numpy().view(np.uint16).astype(np.int32)
+    assert idxn.max() < w.K
+    assert np.array_equal(What.numpy().view(np.uint16), oracle.decode(C16n, idxn, d_out, d_in).view(np.uint16))
+    err = ((W.astype(np.float64) - What.numpy().astype(np.float64)) ** 2).sum()
+    # padded coordinates are ordinary zeros for the clustering: they add the square of the chosen centroid's
+    # coordinate to the objective but are dropped by decode
+    pad = (-d_out) % w.g
+    rec = C16n.astype(np.float64)[idxn].reshape(d_in, -1)          # (in_features, out_pad)
+    pad_share = (rec[:, d_out:] ** 2).sum() if pad else 0.0
+    assert pad > 0 and pad_share > 0
+    assert tr[-1].item() == pytest.approx(err + pad_share, rel=1e-7)   # dist is rounded to FP32 per point
+    u.check_assign_against_oracle(X, C16n.astype(np.float32), idxn, None, sel)
+
+
 def test_cfg4_full_size_one_iteration_sampled():
     u = _u()
     w = wl.WORKLOADS["cfg4_8192x28672_g4_k65536"]

@@ -28,37 +28,36 @@ reshape_transpose_kernel(const uint16_t* __restrict__ W, int64_t d_out, int64_t 
 }
 
 // ---- 16-byte versions of the two transposing kernels (taken when every row is a whole number of
-// 8-element groups).  A 64 x 64 tile goes through shared memory with a row stride of 33 words:
-// global reads and writes are 16-byte vectors along the contiguous axis of each side, and the
-// column reads in shared memory spread over the banks.
-constexpr int TSW = 33;   // tile row stride in 32-bit words (64 halves + 2)
+// 8-element groups).  A 64 x 64 tile goes through shared memory as 32-bit words (two elements),
+// row r at word offset 33 r + 4 (r / 32): with that stride both the row-wise writes (four words per
+// thread) and the column-wise reads (one word from each of eight rows) touch 32 different banks
+// per warp.  A thread of the second phase reads eight words, i.e. a 8 x 2 block, and writes two
+// 16-byte vectors into two adjacent output rows.
+constexpr int TILE_WORDS = TD * 33 + 4;
 
-// Writes the transposed tile: output row `ro` (0..63) takes element [8c+k][ro], k = 0..7, as one vector.
-__device__ __forceinline__ uint4 tile_column8(const unsigned* tile, int c, int ro) {
-    unsigned short h[8];
-#pragma unroll
-    for (int k = 0; k < 8; ++k) {
-        const unsigned w = tile[(8 * c + k) * TSW + (ro >> 1)];
-        h[k] = (ro & 1) ? (unsigned short)(w >> 16) : (unsigned short)(w & 0xffffu);
-    }
-    uint4 v;
-    v.x = (unsigned)h[0] | ((unsigned)h[1] << 16);
-    v.y = (unsigned)h[2] | ((unsigned)h[3] << 16);
-    v.z = (unsigned)h[4] | ((unsigned)h[5] << 16);
-    v.w = (unsigned)h[6] | ((unsigned)h[7] << 16);
-    return v;
-}
+__device__ __forceinline__ int tile_row(int r) { return r * 33 + (r >> 5) * 4; }
 
 __device__ __forceinline__ void tile_put8(unsigned* tile, int r, int c, uint4 v) {
-    unsigned* dst = tile + r * TSW + 4 * c;
+    unsigned* dst = tile + tile_row(r) + 4 * c;
     dst[0] = v.x; dst[1] = v.y; dst[2] = v.z; dst[3] = v.w;
+}
+
+// Elements [8c+k][2rp] (k = 0..7) into `even`, [8c+k][2rp+1] into `odd`.
+__device__ __forceinline__ void tile_column8x2(const unsigned* tile, int c, int rp, uint4& even, uint4& odd) {
+    unsigned w[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) w[k] = tile[tile_row(8 * c + k) + rp];
+    even.x = __byte_perm(w[0], w[1], 0x5410); odd.x = __byte_perm(w[0], w[1], 0x7632);
+    even.y = __byte_perm(w[2], w[3], 0x5410); odd.y = __byte_perm(w[2], w[3], 0x7632);
+    even.z = __byte_perm(w[4], w[5], 0x5410); odd.z = __byte_perm(w[4], w[5], 0x7632);
+    even.w = __byte_perm(w[6], w[7], 0x5410); odd.w = __byte_perm(w[6], w[7], 0x7632);
 }
 
 // PAPER_T reshape; needs d_in % 8 == 0 and out_pad % 8 == 0.
 __global__ void __launch_bounds__(256)
 reshape_transpose_vec_kernel(const uint16_t* __restrict__ W, int64_t d_out, int64_t d_in, int64_t out_pad,
                              uint16_t* __restrict__ X) {
-    __shared__ unsigned tile[TD * TSW];
+    __shared__ unsigned tile[TILE_WORDS];
     const int64_t i0 = (int64_t)blockIdx.x * TD, o0 = (int64_t)blockIdx.y * TD;
     const int c = threadIdx.x & 7, r0 = threadIdx.x >> 3;
 #pragma unroll
@@ -70,11 +69,14 @@ reshape_transpose_vec_kernel(const uint16_t* __restrict__ W, int64_t d_out, int6
         tile_put8(tile, r, c, v);
     }
     __syncthreads();
-#pragma unroll
-    for (int p = 0; p < 2; ++p) {               // rows: in_features, vectors along out_features
-        const int r = r0 + 32 * p;
-        const int64_t i = i0 + r, o = o0 + 8 * c;
-        if (i < d_in && o < out_pad) *reinterpret_cast<uint4*>(X + i * out_pad + o) = tile_column8(tile, c, r);
+    {                                           // rows: in_features 2 r0, 2 r0 + 1, vectors along out_features
+        uint4 even, odd;
+        tile_column8x2(tile, c, r0, even, odd);
+        const int64_t i = i0 + 2 * r0, o = o0 + 8 * c;
+        if (o < out_pad) {
+            if (i < d_in) *reinterpret_cast<uint4*>(X + i * out_pad + o) = even;
+            if (i + 1 < d_in) *reinterpret_cast<uint4*>(X + (i + 1) * out_pad + o) = odd;
+        }
     }
 }
 
@@ -85,7 +87,7 @@ template <int G>
 __global__ void __launch_bounds__(256)
 decode_transpose_vec_kernel(const uint16_t* __restrict__ C16, const uint16_t* __restrict__ idx, int64_t d_out,
                             int64_t d_in, int64_t out_pad, uint16_t* __restrict__ W_hat) {
-    __shared__ unsigned tile[TD * TSW];
+    __shared__ unsigned tile[TILE_WORDS];
     const int64_t i0 = (int64_t)blockIdx.x * TD, o0 = (int64_t)blockIdx.y * TD;
     const int c = threadIdx.x & 7, r0 = threadIdx.x >> 3;
 #pragma unroll
@@ -96,9 +98,10 @@ decode_transpose_vec_kernel(const uint16_t* __restrict__ C16, const uint16_t* __
         if (i < d_in && o < out_pad) {
             const int64_t flat = i * out_pad + o;
             const int64_t n = flat / G;
-            if constexpr (G == 4) {
-                const uint2 a = __ldg(reinterpret_cast<const uint2*>(C16 + (int64_t)__ldg(idx + n) * 4));
-                const uint2 b = __ldg(reinterpret_cast<const uint2*>(C16 + (int64_t)__ldg(idx + n + 1) * 4));
+            if constexpr (G == 4) {             // flat is a multiple of 8: n is even, both codes in one word
+                const unsigned two = __ldg(reinterpret_cast<const unsigned*>(idx + n));
+                const uint2 a = __ldg(reinterpret_cast<const uint2*>(C16 + (int64_t)(two & 0xffffu) * 4));
+                const uint2 b = __ldg(reinterpret_cast<const uint2*>(C16 + (int64_t)(two >> 16) * 4));
                 v = make_uint4(a.x, a.y, b.x, b.y);
             } else {
                 v = __ldg(reinterpret_cast<const uint4*>(C16 + (int64_t)__ldg(idx + n) * G + (flat - n * G)));
@@ -107,11 +110,14 @@ decode_transpose_vec_kernel(const uint16_t* __restrict__ C16, const uint16_t* __
         tile_put8(tile, r, c, v);
     }
     __syncthreads();
-#pragma unroll
-    for (int p = 0; p < 2; ++p) {               // rows: out_features, vectors along in_features
-        const int r = r0 + 32 * p;
-        const int64_t o = o0 + r, i = i0 + 8 * c;
-        if (o < d_out && i < d_in) *reinterpret_cast<uint4*>(W_hat + o * d_in + i) = tile_column8(tile, c, r);
+    {                                           // rows: out_features 2 r0, 2 r0 + 1, vectors along in_features
+        uint4 even, odd;
+        tile_column8x2(tile, c, r0, even, odd);
+        const int64_t o = o0 + 2 * r0, i = i0 + 8 * c;
+        if (i < d_in) {
+            if (o < d_out) *reinterpret_cast<uint4*>(W_hat + o * d_in + i) = even;
+            if (o + 1 < d_out) *reinterpret_cast<uint4*>(W_hat + (o + 1) * d_in + i) = odd;
+        }
     }
 }
 

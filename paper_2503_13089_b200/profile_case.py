@@ -45,20 +45,26 @@ def main():
     W = torch.empty((d_out, d_in), dtype=torch.float16, device="cuda")
     cc.cc_assign(ctx, X, N, g, C, K, idx, dist, obj, nres)      # warm-up; also valid codes for update / decode
     cc.cc_finalize(ctx, X, N, g, C, K, C16, idx, dist, obj)
+    def once():
+        if a.kernel == "assign":
+            cc.cc_assign(ctx, X, N, g, C, K, idx, dist, obj, nres)
+        elif a.kernel == "update":
+            cc.cc_update(ctx, X, N, g, idx, K, C2, counts)
+        elif a.kernel == "decode":
+            cc.cc_decode(ctx, C16, K, g, idx, d_out, d_in, cc.LAYOUT_PAPER_T, W)
+        elif a.kernel == "reshape":
+            cc.cc_reshape_subvectors(ctx, W, d_out, d_in, g, cc.LAYOUT_PAPER_T, X2)
+        else:
+            cc.cc_fit(ctx, X, N, g, K, a.iters, C, idx, dist, counts, None)
+
+    C2 = C.clone()
+    X2 = torch.empty_like(X)
+    once()                                   # untimed: the first launch of a kernel also loads it
     torch.cuda.synchronize()
     cc.cc_profile_enable(ctx, True)
     cc.cc_profile_read(ctx)
     for _ in range(a.reps):
-        if a.kernel == "assign":
-            cc.cc_assign(ctx, X, N, g, C, K, idx, dist, obj, nres)
-        elif a.kernel == "update":
-            cc.cc_update(ctx, X, N, g, idx, K, C, counts)
-        elif a.kernel == "decode":
-            cc.cc_decode(ctx, C16, K, g, idx, d_out, d_in, cc.LAYOUT_PAPER_T, W)
-        elif a.kernel == "reshape":
-            cc.cc_reshape_subvectors(ctx, W, d_out, d_in, g, cc.LAYOUT_PAPER_T, X)
-        else:
-            cc.cc_fit(ctx, X, N, g, K, a.iters, C, idx, dist, counts, None)
+        once()
     torch.cuda.synchronize()
     prof = cc.cc_profile_read(ctx)
     cc.cc_poll_status(ctx)

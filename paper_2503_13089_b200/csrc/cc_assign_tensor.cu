@@ -276,11 +276,15 @@ prep_rescan_kernel(const float* __restrict__ C, int K, int Kpad, float* __restri
 
 // DUMP = true writes every score (divided by S) to `dump` (row stride dump_ld) instead of
 // reducing them: a verification aid for the rounding model, used on small inputs only.
-template <int G, bool DUMP>
+// FULL = true: every CTA of the launch holds exactly NA point tiles, which makes the accumulator
+// slot and the barrier phase of tile (b, a) compile-time functions of a; the ragged rest of the
+// points (and small inputs) go through FULL = false, starting at point tile `tile_offset`.
+template <int G, bool DUMP, bool FULL>
 __global__ void __launch_bounds__(TC_THREADS, 1)
 assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* __restrict__ gB, int n_btiles,
-                     int na_per_cta, const TcParams* __restrict__ params, float2* __restrict__ tstate,
-                     unsigned* __restrict__ status, float* __restrict__ dump, int64_t dump_ld) {
+                     int na_per_cta, int64_t tile_offset, const TcParams* __restrict__ params,
+                     float2* __restrict__ tstate, unsigned* __restrict__ status, float* __restrict__ dump,
+                     int64_t dump_ld) {
     using Cfg = TcCfg<G>;
     constexpr int KD = Cfg::KD, SPLIT = Cfg::SPLIT, STAGES = Cfg::STAGES;
     constexpr int A_TILE = Cfg::A_TILE, B_TILE = Cfg::B_TILE;
@@ -294,9 +298,9 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* 
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int64_t tile0 = (int64_t)blockIdx.x * na_per_cta;          // first point tile of this CTA
+    const int64_t tile0 = tile_offset + (int64_t)blockIdx.x * na_per_cta;   // first point tile of this CTA
     const int64_t n_tiles = (N + TM - 1) / TM;
-    const int na = (int)((n_tiles - tile0 < na_per_cta) ? (n_tiles - tile0) : na_per_cta);
+    const int na = FULL ? NA : (int)((n_tiles - tile0 < na_per_cta) ? (n_tiles - tile0) : na_per_cta);
     const int64_t base = tile0 * TM;
 
     if (tid == 0) {
@@ -386,9 +390,14 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* 
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint64_t descB = descB0 + (uint64_t)((st * B_TILE) >> 4);
-                for (int a = 0; a < na; ++a, ++q) {
-                    const int slot = q % SLOTS;
-                    ok = mbar_wait(smem_u32(t_empty + slot), ((q / SLOTS) & 1) ^ 1, abort_flag);
+#pragma unroll
+                for (int a = 0; a < NA; ++a) {
+                    if (a >= na) break;
+                    // with NA = 8 tiles per codebook tile the slot and phase of tile (b, a) depend on a only
+                    const int slot = FULL ? (a % SLOTS) : (q % SLOTS);
+                    const uint32_t par = FULL ? ((a / SLOTS) & 1) : ((q / SLOTS) & 1);
+                    ++q;
+                    ok = mbar_wait(smem_u32(t_empty + slot), par ^ 1, abort_flag);
                     if (!ok) break;
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     const uint64_t descA = descA0 + (uint64_t)((a * A_TILE) >> 4);
@@ -426,12 +435,14 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* 
         const uint32_t tbase = tmem + ((uint32_t)(quarter * 32) << 16) + cg * TCHUNK;
         bool ok = true;
         int q = 0;
-        for (int b = 0; b < n_btiles && ok; ++b) {
+        int chunk_id = cg;                                // id of this warp's chunk in codebook tile b
+        for (int b = 0; b < n_btiles && ok; ++b, chunk_id += EW) {
 #pragma unroll
             for (int a = 0; a < NA; ++a) {
                 if (a >= na || !ok) continue;
-                const int slot = q % SLOTS;
-                ok = mbar_wait(smem_u32(t_full + slot), (q / SLOTS) & 1, abort_flag);
+                const int slot = FULL ? (a % SLOTS) : (q % SLOTS);
+                const uint32_t par = FULL ? ((a / SLOTS) & 1) : ((q / SLOTS) & 1);
+                ok = mbar_wait(smem_u32(t_full + slot), par, abort_flag);
                 ++q;
                 if (!ok) continue;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
@@ -481,7 +492,6 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* 
                         m2 = min3(m2, __uint_as_float(v[23]), __uint_as_float(v[31]));
                     }
                     const float m = fminf(min3(m0, m1, m2), m3);
-                    const int chunk_id = b * EW + cg;
                     const bool better = m < b1[a];
                     b2[a] = better ? b1[a] : fminf(b2[a], m);
                     bc[a] = better ? chunk_id : bc[a];
@@ -649,29 +659,33 @@ cudaError_t launch_tensor(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int
         const int64_t n_tiles = (N + TM - 1) / TM;
         int64_t na_per_cta = (n_tiles + ctx->sm_count - 1) / ctx->sm_count;    // small inputs still use every SM
         if (na_per_cta > NA) na_per_cta = NA;
-        const int64_t blocks = (n_tiles + na_per_cta - 1) / na_per_cta;
-        if (dump) {
-            static bool attr_set = false;
-            if (!attr_set) {
-                e = cudaFuncSetAttribute(assign_tensor_kernel<G, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
-                if (e != cudaSuccess) return e;
-                attr_set = true;
-            }
-            ProfScope ps(ctx, CC_K_OTHER, st);
-            assign_tensor_kernel<G, true><<<(unsigned)blocks, TC_THREADS, Cfg::SMEM, st>>>(
-                X, N, gB, Kpad / TN, (int)na_per_cta, params, tstate, status, dump, dump_ld);
-            return cudaGetLastError();
-        }
         static bool attr_set = false;
         if (!attr_set) {
-            e = cudaFuncSetAttribute(assign_tensor_kernel<G, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM);
-            if (e != cudaSuccess) return e;
+            if ((e = cudaFuncSetAttribute(assign_tensor_kernel<G, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM)) != cudaSuccess) return e;
+            if ((e = cudaFuncSetAttribute(assign_tensor_kernel<G, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM)) != cudaSuccess) return e;
+            if ((e = cudaFuncSetAttribute(assign_tensor_kernel<G, false, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM)) != cudaSuccess) return e;
             attr_set = true;
+        }
+        if (dump) {
+            const int64_t blocks = (n_tiles + na_per_cta - 1) / na_per_cta;
+            ProfScope ps(ctx, CC_K_OTHER, st);
+            assign_tensor_kernel<G, true, false><<<(unsigned)blocks, TC_THREADS, Cfg::SMEM, st>>>(
+                X, N, gB, Kpad / TN, (int)na_per_cta, 0, params, tstate, status, dump, dump_ld);
+            return cudaGetLastError();
         }
         {
             ProfScope ps(ctx, CC_K_ASSIGN_MAIN, st);
-            assign_tensor_kernel<G, false><<<(unsigned)blocks, TC_THREADS, Cfg::SMEM, st>>>(
-                X, N, gB, Kpad / TN, (int)na_per_cta, params, tstate, status, nullptr, 0);
+            // CTAs with a full set of NA point tiles, then the ragged rest
+            const int64_t full_blocks = (na_per_cta == NA) ? n_tiles / NA : 0;
+            if (full_blocks > 0)
+                assign_tensor_kernel<G, false, true><<<(unsigned)full_blocks, TC_THREADS, Cfg::SMEM, st>>>(
+                    X, N, gB, Kpad / TN, NA, 0, params, tstate, status, nullptr, 0);
+            const int64_t rest_tiles = n_tiles - full_blocks * NA;
+            if (rest_tiles > 0) {
+                const int64_t blocks = (rest_tiles + na_per_cta - 1) / na_per_cta;
+                assign_tensor_kernel<G, false, false><<<(unsigned)blocks, TC_THREADS, Cfg::SMEM, st>>>(
+                    X, N, gB, Kpad / TN, (int)na_per_cta, full_blocks * NA, params, tstate, status, nullptr, 0);
+            }
         }
         {
             ProfScope ps(ctx, CC_K_ASSIGN_FINISH, st);

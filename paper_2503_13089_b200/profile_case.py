@@ -41,7 +41,8 @@ def main():
     nres = torch.zeros(1, dtype=torch.int64, device="cuda")
     C16 = torch.empty((K, g), dtype=torch.float16, device="cuda")
     d_out, d_in = g * 1024, N // 1024
-    assert d_in * 1024 == N, "N must be a multiple of 1024 for the reshape / decode cases"
+    if a.kernel in ("decode", "reshape"):
+        assert d_in * 1024 == N, "N must be a multiple of 1024 for the reshape / decode cases"
     W = torch.empty((d_out, d_in), dtype=torch.float16, device="cuda")
     cc.cc_assign(ctx, X, N, g, C, K, idx, dist, obj, nres)      # warm-up; also valid codes for update / decode
     cc.cc_finalize(ctx, X, N, g, C, K, C16, idx, dist, obj)

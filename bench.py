@@ -387,7 +387,7 @@ def main():
             "ms_steps": ms_steps,
             "e2e": {"value": total_evals / (e2e_step * 1e-3), "unit": "distance evaluations/s",
                     "ms_per_step": e2e_step, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
-                    "api": "cc_compress_host (pinned host buffers in and out, allocation included)"},
+                    "api": "cc_compress_host (pinned host buffers in and out; its device buffer is allocated by the untimed first call)"},
             "gpu_launches": launches,
             "roofline": roofline,
             "kernels": kern,

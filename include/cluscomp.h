@@ -25,7 +25,7 @@
  *  - The same inputs give bit-identical outputs on every call.
  *  - Scratch memory is one caller-owned workspace (cc_workspace_bytes /
  *    cc_set_workspace); the library itself allocates no device memory except
- *    in cc_compress_host.
+ *    in cc_compress_host (a buffer kept in the context).
  */
 #ifndef CLUSCOMP_H_
 #define CLUSCOMP_H_
@@ -68,7 +68,7 @@ typedef enum {
 typedef struct cc_ctx cc_ctx; /* opaque; one per device and per concurrent user */
 
 /* Context.  cc_create binds to `device` (cudaSetDevice is called inside every entry point).
- * cc_destroy frees only host state; the workspace stays the caller's. */
+ * cc_destroy frees host state and the buffer of cc_compress_host; the workspace stays the caller's. */
 cc_status cc_create(cc_ctx** out, int device);
 cc_status cc_destroy(cc_ctx* ctx);
 const char* cc_status_string(cc_status s);
@@ -215,7 +215,8 @@ cc_status cc_poll_status(cc_ctx* ctx, void* stream);
 /* Whole path on HOST buffers (Sections 3.1-3.2 end to end): copies W to the device, reshapes,
  * initialises, runs `iters` Lloyd iterations, finalises, and copies the FP16 codebook, the
  * codes and the final objective back; optionally also decodes into W_hat_host (may be NULL).
- * Allocates and frees its own device buffers and workspace and synchronises before returning.
+ * Uses a device buffer of its own that the context keeps and grows on demand (the first call of a
+ * size allocates, later calls do not; cc_destroy frees it) and synchronises before returning.
  * All pointers are host pointers (pinned memory makes the copies asynchronous).
  * objective_trace_host (may be NULL): iters + 1 doubles, the last being the final objective. */
 cc_status cc_compress_host(cc_ctx* ctx, const uint16_t* W_host, int64_t d_out, int64_t d_in, int g,

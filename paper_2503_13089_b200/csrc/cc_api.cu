@@ -129,6 +129,8 @@ cc_status cc_create(cc_ctx** out, int device) {
     c->prof_on = 0;
     c->prof_used = c->prof_made = 0;
     c->prof = nullptr;
+    c->e2e_buf = nullptr;
+    c->e2e_bytes = 0;
     *out = c;
     return CC_OK;
 }
@@ -136,6 +138,10 @@ cc_status cc_create(cc_ctx** out, int device) {
 cc_status cc_destroy(cc_ctx* ctx) {
     if (!ctx) return CC_ERR_NULL;
     delete[] ctx->pos_host;
+    if (ctx->e2e_buf) {
+        cudaSetDevice(ctx->device);
+        cudaFree(ctx->e2e_buf);
+    }
     if (ctx->prof) {
         cudaSetDevice(ctx->device);
         for (int i = 0; i < ctx->prof_made; ++i) { cudaEventDestroy(ctx->prof[i].a); cudaEventDestroy(ctx->prof[i].b); }
@@ -360,8 +366,14 @@ cc_status cc_compress_host(cc_ctx* ctx, const uint16_t* W_host, int64_t d_out, i
     const size_t oW = take(w_bytes), oX = take(x_bytes), oC = take((size_t)K * g * 4), oC16 = take((size_t)K * g * 2),
                  oIdx = take((size_t)N * 2), oDist = take((size_t)N * 4), oCnt = take((size_t)K * 4),
                  oTr = take((size_t)(iters + 1) * 8), oWs = take(ws_bytes);
-    char* base = nullptr;
-    if (cudaMalloc(&base, off) != cudaSuccess) return CC_ERR_CUDA;
+    if (ctx->e2e_bytes < off) {          // grown on demand and kept: repeated calls allocate nothing
+        if (ctx->e2e_buf) cudaFree(ctx->e2e_buf);
+        ctx->e2e_buf = nullptr;
+        ctx->e2e_bytes = 0;
+        if (cudaMalloc(&ctx->e2e_buf, off) != cudaSuccess) return CC_ERR_CUDA;
+        ctx->e2e_bytes = off;
+    }
+    char* base = static_cast<char*>(ctx->e2e_buf);
     void* saved_ws = ctx->ws;
     const size_t saved_bytes = ctx->ws_bytes;
     cc_status s = cc_set_workspace(ctx, base + oWs, ws_bytes);
@@ -394,7 +406,6 @@ cc_status cc_compress_host(cc_ctx* ctx, const uint16_t* W_host, int64_t d_out, i
     else cudaStreamSynchronize(st);
     ctx->ws = saved_ws;
     ctx->ws_bytes = saved_bytes;
-    cudaFree(base);
     return s;
 }
 

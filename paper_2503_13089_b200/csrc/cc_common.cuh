@@ -30,6 +30,8 @@ struct cc_ctx {
     int prof_on;          // record an event pair around every kernel launch
     int prof_used, prof_made;
     cc_prof_slot* prof;   // CC_PROF_CAP slots, events created on first use
+    void* e2e_buf;        // device memory of cc_compress_host, grown on demand, freed by cc_destroy
+    size_t e2e_bytes;
 };
 
 // Brackets one kernel launch with events on its stream when timing is enabled, and counts it.

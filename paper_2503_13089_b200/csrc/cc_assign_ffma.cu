@@ -240,12 +240,27 @@ assign_ffma_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __res
 }
 
 // ---------------------------------------------------------------------------------------------
-// Exact stage.  Each flagged point is scanned against every centroid by a group of T threads
-// (T = 128, 32, 8 or 1, chosen from the number of flagged points so that few points still fill
-// the GPU and many points do not re-read the codebook too often).  A cheap FP32 direct-form
-// distance (relative error <= (g+2) 2^-24, no cancellation) screens the candidates; those within
-// 2^-18 of the best FP64 distance so far are recomputed in FP64 (sub, mul, add, in dimension
-// order, no FMA contraction) and the pair (distance, index) is minimised lexicographically.
+// Exact stage.  Every flagged point is scanned against every centroid again, the codebook being
+// cut into S slices so that (point, slice) items fill the GPU whether few or many points are
+// flagged (S is derived on the device from the number of flagged points; consecutive threads take
+// consecutive points of the same slice, so a warp reads each centroid once for 32 points).
+// A cheap FP32 direct-form distance (relative error <= (g+2) 2^-24, no cancellation) screens the
+// candidates; those within 2^-18 of the best FP64 distance so far are recomputed in FP64 (sub,
+// mul, add, in dimension order, no FMA contraction) and the pair (distance, index) is minimised
+// lexicographically.  Each item starts from the fast stage's winner, writes its slice's result to
+// scratch, and a second kernel merges the S results of a point (one warp per point).
+struct ResolveEntry { double D; int j; int pad; };
+
+__device__ __forceinline__ int resolve_slices(ull F, ull total_threads, int K, int64_t cap_entries) {
+    ull S = (2 * total_threads + F - 1) / F;
+    ull smax = (ull)(K >= 16 ? K / 8 : 1);
+    if (smax > 256) smax = 256;
+    const ull by_cap = (ull)cap_entries / F;
+    if (smax > by_cap) smax = by_cap;
+    if (S > smax) S = smax;
+    return S < 1 ? 1 : (int)S;
+}
+
 template <int G>
 __device__ __forceinline__ void load_centroid(const float* __restrict__ C, int j, float* c) {
     const float* row = C + (int64_t)j * G;
@@ -263,26 +278,21 @@ __device__ __forceinline__ void load_centroid(const float* __restrict__ C, int j
 
 template <int G>
 __global__ void __launch_bounds__(128)
-resolve_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restrict__ C, int K,
-               const unsigned* __restrict__ status, const unsigned* __restrict__ flagged,
-               uint16_t* __restrict__ idx, float* __restrict__ dist) {
-    __shared__ double sh_d[4];
-    __shared__ int sh_j[4];
+resolve_scan_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restrict__ C, int K,
+                    const unsigned* __restrict__ status, const unsigned* __restrict__ flagged,
+                    ResolveEntry* __restrict__ scratch, int64_t cap_entries, uint16_t* __restrict__ idx,
+                    float* __restrict__ dist) {
     ull F = *reinterpret_cast<const ull*>(status + 2);
     if (F > (ull)N) F = (ull)N;
     if (F == 0) return;
     const ull total_threads = (ull)gridDim.x * blockDim.x;
-    // threads per point: a whole block while the flagged points are fewer than the blocks, then a
-    // warp, 8 lanes, one lane
-    const int T = (F <= (ull)gridDim.x) ? 128 : (F * 32 <= total_threads) ? 32 : (F * 8 <= total_threads) ? 8 : 1;
-    const ull gthread = (ull)blockIdx.x * blockDim.x + threadIdx.x;
-    const int lane = (int)(gthread % T);
-    const ull n_groups = total_threads / T;
-    const ull n_rounds = (F + n_groups - 1) / n_groups;       // the same for every thread of a block
-    for (ull r = 0; r < n_rounds; ++r) {
-        const ull f = r * n_groups + gthread / T;
-        const bool live = f < F;
-        const int64_t i = live ? flagged[f] : 0;
+    const int S = resolve_slices(F, total_threads, K, cap_entries);
+    const int L = (K + S - 1) / S;
+    const ull items = F * (ull)S;
+    for (ull item = (ull)blockIdx.x * blockDim.x + threadIdx.x; item < items; item += total_threads) {
+        const int sl = (int)(item / F);
+        const ull f = item - (ull)sl * F;
+        const int64_t i = flagged[f];
         float x[G];
         bool nf = false;
         load_point<G>(X, i, N, x, nf);
@@ -294,9 +304,9 @@ resolve_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restric
             Db = __dadd_rn(Db, __dmul_rn(df, df));
         }
         float bound = __double2float_ru(Db * (1.0 + 3.814697265625e-6));
-        const int k_end = live ? K : 0;        // idle groups skip the scan
+        const int j_end = (sl + 1) * L < K ? (sl + 1) * L : K;
 #pragma unroll 2
-        for (int j = lane; j < k_end; j += T) {
+        for (int j = sl * L; j < j_end; ++j) {
             float c[G];
             load_centroid<G>(C, j, c);
             float dh = 0.f;
@@ -315,26 +325,43 @@ resolve_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restric
                 }
             }
         }
-        // lexicographic minimum of (distance, index) over the T threads of the group
-        const int TW = T > 32 ? 32 : T;
-        for (int o = TW >> 1; o > 0; o >>= 1) {
+        if (S == 1) {            // one item per point: nothing to merge
+            idx[i] = (uint16_t)jb;
+            dist[i] = (float)Db;
+        } else {
+            ResolveEntry e;
+            e.D = Db; e.j = jb; e.pad = 0;
+            scratch[(ull)sl * F + f] = e;
+        }
+    }
+}
+
+__global__ void __launch_bounds__(128)
+resolve_merge_kernel(int64_t N, int K, const unsigned* __restrict__ status, const unsigned* __restrict__ flagged,
+                     const ResolveEntry* __restrict__ scratch, int64_t cap_entries, ull scan_threads,
+                     uint16_t* __restrict__ idx, float* __restrict__ dist) {
+    ull F = *reinterpret_cast<const ull*>(status + 2);
+    if (F > (ull)N) F = (ull)N;
+    if (F == 0) return;
+    const int S = resolve_slices(F, scan_threads, K, cap_entries);
+    if (S == 1) return;
+    const int lane = threadIdx.x & 31;
+    const ull n_warps = ((ull)gridDim.x * blockDim.x) >> 5;
+    for (ull f = ((ull)blockIdx.x * blockDim.x + threadIdx.x) >> 5; f < F; f += n_warps) {
+        double Db = INFINITY;
+        int jb = 0x7fffffff;
+        for (int sl = lane; sl < S; sl += 32) {
+            const ResolveEntry e = scratch[(ull)sl * F + f];
+            if (e.D < Db || (e.D == Db && e.j < jb)) { Db = e.D; jb = e.j; }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
             const double Do = __shfl_xor_sync(0xffffffffu, Db, o);
             const int jo = __shfl_xor_sync(0xffffffffu, jb, o);
             if (Do < Db || (Do == Db && jo < jb)) { Db = Do; jb = jo; }
         }
-        if (T == 128) {                         // uniform over the grid
-            const int w = threadIdx.x >> 5;
-            __syncthreads();                    // the previous round's readers are done
-            if ((threadIdx.x & 31) == 0) { sh_d[w] = Db; sh_j[w] = jb; }
-            __syncthreads();
-#pragma unroll
-            for (int o = 0; o < 4; ++o) {
-                const double Do = sh_d[o];
-                const int jo = sh_j[o];
-                if (Do < Db || (Do == Db && jo < jb)) { Db = Do; jb = jo; }
-            }
-        }
-        if (live && lane == 0) {
+        if (lane == 0) {
+            const int64_t i = flagged[f];
             idx[i] = (uint16_t)jb;
             dist[i] = (float)Db;
         }
@@ -413,8 +440,16 @@ cudaError_t launch_tail(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64
     unsigned* flagged = reinterpret_cast<unsigned*>(ws + L.flagged);
     double* partials = reinterpret_cast<double*>(ws + L.partials);
     if (N > 0) {
+        // scratch of the exact stage: the tensor scan's per-point state, free again by now
+        ResolveEntry* scratch = reinterpret_cast<ResolveEntry*>(ws + L.tstate);
+        const int64_t cap_entries = N / 2 > 0 ? N / 2 : 1;
+        const int blocks = ctx->sm_count * 16;
+        {
+            ProfScope ps(ctx, CC_K_RESOLVE, st);
+            resolve_scan_kernel<G><<<blocks, 128, 0, st>>>(X, N, C, K, status, flagged, scratch, cap_entries, idx, dist);
+        }
         ProfScope ps(ctx, CC_K_RESOLVE, st);
-        resolve_kernel<G><<<ctx->sm_count * 16, 128, 0, st>>>(X, N, C, K, status, flagged, idx, dist);
+        resolve_merge_kernel<<<blocks, 128, 0, st>>>(N, K, status, flagged, scratch, cap_entries, (ull)blocks * 128, idx, dist);
     }
     if (objective || n_resolved) {
         int blocks = (int)((N + 4095) / 4096);

@@ -274,6 +274,69 @@ prep_rescan_kernel(const float* __restrict__ C, int K, int Kpad, float* __restri
                    "+r"(v[29]), "+r"(v[30]), "+r"(v[31])                                                         \
                  :: "memory")
 
+// A operand rows [x repeated SPLIT times, 2^15, 2^6, 2^-3, 2^-12, 0..] of points base + e,
+// e = first, first + step, .. < count, into the tiles at sA (canonical layout, 16 bytes at a time).
+template <int G>
+__device__ __forceinline__ void build_a_rows(const uint16_t* __restrict__ X, int64_t N, int64_t base, int first,
+                                             int step, int count, unsigned char* sA, bool& nonfinite) {
+    using Cfg = TcCfg<G>;
+    constexpr int KD = Cfg::KD, SPLIT = Cfg::SPLIT;
+    for (int e = first; e < count; e += step) {
+        float x[G];
+        load_point<G>(X, base + e, N, x, nonfinite);
+        unsigned short h[KD];
+#pragma unroll
+        for (int k = 0; k < KD; ++k) {
+            h[k] = (k < SPLIT * G) ? __half_as_ushort(__float2half_rn(x[k % G]))    // exact: x is FP16 data
+                 : (k < SPLIT * G + NQ) ? __half_as_ushort(__float2half_rn(qconst(k - SPLIT * G)))
+                 : (unsigned short)0;
+        }
+        unsigned char* tile = sA + (e / TM) * Cfg::A_TILE;
+        const int r = e % TM;
+#pragma unroll
+        for (int kc = 0; kc < KD / 8; ++kc) {
+            uint4 w;
+            w.x = (unsigned)h[kc * 8 + 0] | ((unsigned)h[kc * 8 + 1] << 16);
+            w.y = (unsigned)h[kc * 8 + 2] | ((unsigned)h[kc * 8 + 3] << 16);
+            w.z = (unsigned)h[kc * 8 + 4] | ((unsigned)h[kc * 8 + 5] << 16);
+            w.w = (unsigned)h[kc * 8 + 6] | ((unsigned)h[kc * 8 + 7] << 16);
+            *reinterpret_cast<uint4*>(tile + canon_bytes(r, kc * 8, TM)) = w;
+        }
+    }
+}
+
+// The reduction of one 64-column chunk held in two 32-register halves: four independent chains,
+// 30 three-input minima + 2.
+__device__ __forceinline__ float chunk_min64(const uint32_t* v0, const uint32_t* v1) {
+    float m0 = min3(__uint_as_float(v0[0]), __uint_as_float(v0[1]), __uint_as_float(v0[2]));
+    float m1 = min3(__uint_as_float(v0[8]), __uint_as_float(v0[9]), __uint_as_float(v0[10]));
+    float m2 = min3(__uint_as_float(v0[16]), __uint_as_float(v0[17]), __uint_as_float(v0[18]));
+    float m3 = min3(__uint_as_float(v0[24]), __uint_as_float(v0[25]), __uint_as_float(v0[26]));
+#pragma unroll
+    for (int hf = 0; hf < 2; ++hf) {
+        const uint32_t* v = hf ? v1 : v0;
+        if (hf) {
+            m0 = min3(m0, __uint_as_float(v[0]), __uint_as_float(v[1]));
+            m1 = min3(m1, __uint_as_float(v[8]), __uint_as_float(v[9]));
+            m2 = min3(m2, __uint_as_float(v[16]), __uint_as_float(v[17]));
+            m3 = min3(m3, __uint_as_float(v[24]), __uint_as_float(v[25]));
+            m0 = min3(m0, __uint_as_float(v[2]), __uint_as_float(v[10]));
+            m2 = min3(m2, __uint_as_float(v[18]), __uint_as_float(v[26]));
+        }
+        m0 = min3(m0, __uint_as_float(v[3]), __uint_as_float(v[4]));
+        m1 = min3(m1, __uint_as_float(v[11]), __uint_as_float(v[12]));
+        m2 = min3(m2, __uint_as_float(v[19]), __uint_as_float(v[20]));
+        m3 = min3(m3, __uint_as_float(v[27]), __uint_as_float(v[28]));
+        m0 = min3(m0, __uint_as_float(v[5]), __uint_as_float(v[6]));
+        m1 = min3(m1, __uint_as_float(v[13]), __uint_as_float(v[14]));
+        m2 = min3(m2, __uint_as_float(v[21]), __uint_as_float(v[22]));
+        m3 = min3(m3, __uint_as_float(v[29]), __uint_as_float(v[30]));
+        m0 = min3(m0, __uint_as_float(v[7]), __uint_as_float(v[15]));
+        m2 = min3(m2, __uint_as_float(v[23]), __uint_as_float(v[31]));
+    }
+    return fminf(min3(m0, m1, m2), m3);
+}
+
 // DUMP = true writes every score (divided by S) to `dump` (row stride dump_ld) instead of
 // reducing them: a verification aid for the rounding model, used on small inputs only.
 // FULL = true: every CTA of the launch holds exactly NA point tiles, which makes the accumulator
@@ -286,7 +349,7 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* 
                      float2* __restrict__ tstate, unsigned* __restrict__ status, float* __restrict__ dump,
                      int64_t dump_ld) {
     using Cfg = TcCfg<G>;
-    constexpr int KD = Cfg::KD, SPLIT = Cfg::SPLIT, STAGES = Cfg::STAGES;
+    constexpr int KD = Cfg::KD, STAGES = Cfg::STAGES;
     constexpr int A_TILE = Cfg::A_TILE, B_TILE = Cfg::B_TILE;
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     unsigned char* sA = smem_raw;                                   // NA tiles
@@ -315,30 +378,8 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* 
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
-    // ---- A operand: [x repeated SPLIT times, 2^15, 2^6, 2^-3, 2^-12, 0..] per point, 16 bytes at a time
     bool nonfinite = false;
-    for (int e = tid; e < na * TM; e += TC_THREADS) {
-        float x[G];
-        load_point<G>(X, base + e, N, x, nonfinite);
-        unsigned short h[KD];
-#pragma unroll
-        for (int k = 0; k < KD; ++k) {
-            h[k] = (k < SPLIT * G) ? __half_as_ushort(__float2half_rn(x[k % G]))    // exact: x is FP16 data
-                 : (k < SPLIT * G + NQ) ? __half_as_ushort(__float2half_rn(qconst(k - SPLIT * G)))
-                 : (unsigned short)0;
-        }
-        unsigned char* tile = sA + (e / TM) * A_TILE;
-        const int r = e % TM;
-#pragma unroll
-        for (int kc = 0; kc < KD / 8; ++kc) {
-            uint4 w;
-            w.x = (unsigned)h[kc * 8 + 0] | ((unsigned)h[kc * 8 + 1] << 16);
-            w.y = (unsigned)h[kc * 8 + 2] | ((unsigned)h[kc * 8 + 3] << 16);
-            w.z = (unsigned)h[kc * 8 + 4] | ((unsigned)h[kc * 8 + 5] << 16);
-            w.w = (unsigned)h[kc * 8 + 6] | ((unsigned)h[kc * 8 + 7] << 16);
-            *reinterpret_cast<uint4*>(tile + canon_bytes(r, kc * 8, TM)) = w;
-        }
-    }
+    build_a_rows<G>(X, N, base, tid, TC_THREADS, na * TM, sA, nonfinite);
     if (nonfinite) atomicOr(status, CC_DEV_NONFINITE);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> async proxy (MMA)
     if (warp == 0) {
@@ -464,34 +505,7 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* 
                         for (int u = 0; u < 32; ++u) { row[u] = __uint_as_float(v0[u]) * invS; row[32 + u] = __uint_as_float(v1[u]) * invS; }
                     }
                 } else {
-                    // one chunk of 64 columns, four independent chains (30 three-input minima + 2)
-                    float m0 = min3(__uint_as_float(v0[0]), __uint_as_float(v0[1]), __uint_as_float(v0[2]));
-                    float m1 = min3(__uint_as_float(v0[8]), __uint_as_float(v0[9]), __uint_as_float(v0[10]));
-                    float m2 = min3(__uint_as_float(v0[16]), __uint_as_float(v0[17]), __uint_as_float(v0[18]));
-                    float m3 = min3(__uint_as_float(v0[24]), __uint_as_float(v0[25]), __uint_as_float(v0[26]));
-#pragma unroll
-                    for (int hf = 0; hf < 2; ++hf) {
-                        const uint32_t* v = hf ? v1 : v0;
-                        if (hf) {
-                            m0 = min3(m0, __uint_as_float(v[0]), __uint_as_float(v[1]));
-                            m1 = min3(m1, __uint_as_float(v[8]), __uint_as_float(v[9]));
-                            m2 = min3(m2, __uint_as_float(v[16]), __uint_as_float(v[17]));
-                            m3 = min3(m3, __uint_as_float(v[24]), __uint_as_float(v[25]));
-                            m0 = min3(m0, __uint_as_float(v[2]), __uint_as_float(v[10]));
-                            m2 = min3(m2, __uint_as_float(v[18]), __uint_as_float(v[26]));
-                        }
-                        m0 = min3(m0, __uint_as_float(v[3]), __uint_as_float(v[4]));
-                        m1 = min3(m1, __uint_as_float(v[11]), __uint_as_float(v[12]));
-                        m2 = min3(m2, __uint_as_float(v[19]), __uint_as_float(v[20]));
-                        m3 = min3(m3, __uint_as_float(v[27]), __uint_as_float(v[28]));
-                        m0 = min3(m0, __uint_as_float(v[5]), __uint_as_float(v[6]));
-                        m1 = min3(m1, __uint_as_float(v[13]), __uint_as_float(v[14]));
-                        m2 = min3(m2, __uint_as_float(v[21]), __uint_as_float(v[22]));
-                        m3 = min3(m3, __uint_as_float(v[29]), __uint_as_float(v[30]));
-                        m0 = min3(m0, __uint_as_float(v[7]), __uint_as_float(v[15]));
-                        m2 = min3(m2, __uint_as_float(v[23]), __uint_as_float(v[31]));
-                    }
-                    const float m = fminf(min3(m0, m1, m2), m3);
+                    const float m = chunk_min64(v0, v1);
                     const bool better = m < b1[a];
                     b2[a] = better ? b1[a] : fminf(b2[a], m);
                     bc[a] = better ? chunk_id : bc[a];
@@ -529,6 +543,248 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* 
             }
         }
     }
+    if (*abort_flag && lane == 0) atomicOr(status, CC_DEV_TIMEOUT);
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(SLOTS * TN));
+}
+
+// Persistent form of the scan for contraction lengths up to 32 columns (g <= 9): one CTA per SM walks
+// over groups of NA point tiles (group = blockIdx.x, + gridDim.x, ..) and keeps TWO sets of A tiles
+// in shared memory.  A 19th warp builds the next group's A operand while the current group is
+// multiplied and reduced, so the tensor core and the epilogue never wait for a CTA to start or to
+// drain: with few codebook tiles per group (K = 4096: 16) that start-up is a tenth of the time.
+// Roles and barriers are those of assign_tensor_kernel plus a_full / a_empty per A buffer; every
+// group has n_btiles * NA tiles, a multiple of four, so accumulator slot and phase stay
+// compile-time functions of a.
+constexpr int PERSIST_THREADS = TC_THREADS + 32;
+
+template <int G> struct PersistCfg {
+    using Cfg = TcCfg<G>;
+    static constexpr bool OK = Cfg::KD <= 32;
+    static constexpr int SMEM = 2 * NA * Cfg::A_TILE + Cfg::STAGES * Cfg::B_TILE + Cfg::MERGE + 256;
+};
+
+template <int G>
+__global__ void __launch_bounds__(PERSIST_THREADS, 1)
+assign_tensor_persistent_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* __restrict__ gB, int n_btiles,
+                                int n_groups, float2* __restrict__ tstate, unsigned* __restrict__ status) {
+    using Cfg = TcCfg<G>;
+    constexpr int KD = Cfg::KD, STAGES = Cfg::STAGES;
+    constexpr int A_TILE = Cfg::A_TILE, B_TILE = Cfg::B_TILE, A_SET = NA * A_TILE;
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    unsigned char* sA = smem_raw;                                   // 2 sets of NA tiles
+    unsigned char* sB = sA + 2 * A_SET;                             // STAGES tiles
+    float* merge = reinterpret_cast<float*>(sB + STAGES * B_TILE);  // [EW-1][NA][3][TM]
+    uint64_t* bars = reinterpret_cast<uint64_t*>(reinterpret_cast<unsigned char*>(merge) + Cfg::MERGE);
+    uint64_t* b_full = bars, *b_empty = bars + STAGES, *t_full = bars + 2 * STAGES, *t_empty = t_full + SLOTS;
+    uint64_t* a_full = t_empty + SLOTS, *a_empty = a_full + 2;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(a_empty + 2);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int n_iter = (n_groups - (int)blockIdx.x + (int)gridDim.x - 1) / (int)gridDim.x;   // groups of this CTA
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(b_full + s)));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(b_empty + s)));
+        }
+        for (int s = 0; s < SLOTS; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(t_full + s)));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(t_empty + s)), "r"(EPI_WARPS));
+        }
+        for (int s = 0; s < 2; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(a_full + s)));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(a_empty + s)));
+        }
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    // first group's A operand: built by everybody
+    bool nonfinite = false;
+    build_a_rows<G>(X, N, (int64_t)blockIdx.x * (NA * TM), tid, PERSIST_THREADS, NA * TM, sA, nonfinite);
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> async proxy (MMA)
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(SLOTS * TN));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == EPI_WARPS) {
+        // ------------------------------------------------------------ copy warp: B tiles -> ring
+        if (lane == 0) {
+            int st = 0;
+            uint32_t ph = 0;
+            int in_flight_from = 0, total = 0;
+            bool ok = true;
+            for (int it = 0; it < n_iter && ok; ++it) {
+                for (int b = 0; b < n_btiles; ++b) {
+                    if (!mbar_wait(smem_u32(b_empty + st), ph ^ 1, abort_flag)) { ok = false; break; }
+                    const uint32_t bar = smem_u32(b_full + st);
+                    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(B_TILE) : "memory");
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 ::"r"(smem_u32(sB + st * B_TILE)),
+                                   "l"(reinterpret_cast<const unsigned char*>(gB) + (int64_t)b * B_TILE), "r"(B_TILE), "r"(bar)
+                                 : "memory");
+                    ++total;
+                    if (++st == STAGES) { st = 0; ph ^= 1; }
+                }
+            }
+            if (*abort_flag) {   // let the copies in flight land before the CTA exits (bounded)
+                in_flight_from = total > STAGES ? total - STAGES : 0;
+                for (int c = in_flight_from; c < total; ++c) {
+                    const long long t0 = clock64();
+                    while (!mbar_try(smem_u32(b_full + c % STAGES), (c / STAGES) & 1) && clock64() - t0 < WAIT_LIMIT) {}
+                }
+            }
+        }
+    } else if (warp == EPI_WARPS + 1) {
+        // ------------------------------------------------------------ MMA warp: one thread issues
+        if (lane == 0) {
+            const uint32_t idesc = (1u << 4) | ((uint32_t)(TN >> 3) << 17) | ((uint32_t)(TM >> 4) << 24);
+            const uint64_t descA0 = make_desc(smem_u32(sA), TM * 16, 128);
+            const uint64_t descB0 = make_desc(smem_u32(sB), TN * 16, 128);
+            bool ok = true;
+            int st = 0;
+            uint32_t ph = 0;
+            for (int it = 0; it < n_iter && ok; ++it) {
+                const int buf = it & 1;
+                if (it > 0) {      // the first set was built before the barrier above
+                    ok = mbar_wait(smem_u32(a_full + buf), ((it - 1) >> 1) & 1, abort_flag);
+                    if (!ok) break;
+                }
+                for (int b = 0; b < n_btiles && ok; ++b) {
+                    ok = mbar_wait(smem_u32(b_full + st), ph, abort_flag);
+                    if (!ok) break;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    const uint64_t descB = descB0 + (uint64_t)((st * B_TILE) >> 4);
+#pragma unroll
+                    for (int a = 0; a < NA; ++a) {
+                        const int slot = a % SLOTS;
+                        ok = mbar_wait(smem_u32(t_empty + slot), (((a / SLOTS) & 1)) ^ 1, abort_flag);
+                        if (!ok) break;
+                        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                        const uint64_t descA = descA0 + (uint64_t)((buf * A_SET + a * A_TILE) >> 4);
+                        const uint32_t d = tmem + slot * TN;
+#pragma unroll
+                        for (int s = 0; s < KD / 16; ++s) {
+                            const uint64_t da = descA + (uint64_t)((s * 2 * (TM * 16)) >> 4);
+                            const uint64_t db = descB + (uint64_t)((s * 2 * (TN * 16)) >> 4);
+                            if (s == 0)
+                                asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, 0, 0;\n\t"
+                                             "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                                             ::"r"(d), "l"(da), "l"(db), "r"(idesc) : "memory");
+                            else
+                                asm volatile("{\n\t.reg .pred p;\n\tsetp.eq.b32 p, 0, 0;\n\t"
+                                             "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                                             ::"r"(d), "l"(da), "l"(db), "r"(idesc) : "memory");
+                        }
+                        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                                     ::"r"(smem_u32(t_full + slot)) : "memory");
+                    }
+                    if (ok)   // the ring stage may be refilled once these MMAs have read it
+                        asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                                     ::"r"(smem_u32(b_empty + st)) : "memory");
+                    if (++st == STAGES) { st = 0; ph ^= 1; }
+                }
+                if (ok)       // this set of A tiles may be overwritten once the group's MMAs have read it
+                    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                                 ::"r"(smem_u32(a_empty + buf)) : "memory");
+            }
+        }
+    } else if (warp == EPI_WARPS + 2) {
+        // ------------------------------------------------------------ A-operand warp: next group's tiles
+        bool ok = true;
+        for (int it = 1; it < n_iter && ok; ++it) {
+            const int buf = it & 1;
+            if (it >= 2) {     // the set was last used by group it - 2
+                ok = mbar_wait(smem_u32(a_empty + buf), ((it - 2) >> 1) & 1, abort_flag);
+                ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
+                if (!ok) break;
+            }
+            const int64_t group = (int64_t)blockIdx.x + (int64_t)it * gridDim.x;
+            build_a_rows<G>(X, N, group * (NA * TM), lane, 32, NA * TM, sA + buf * A_SET, nonfinite);
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            if (lane == 0)
+                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(a_full + buf)) : "memory");
+        }
+    } else {
+        // ------------------------------------------------------------ epilogue warps
+        const int quarter = warp & 3, cg = warp >> 2;     // TMEM lane quarter, 64-column group
+        const int r = quarter * 32 + lane;                // row of the point tile = TMEM lane
+        const uint32_t tbase = tmem + ((uint32_t)(quarter * 32) << 16) + cg * TCHUNK;
+        bool ok = true;
+        for (int it = 0; it < n_iter && ok; ++it) {
+            float b1[NA], b2[NA];
+            int bc[NA];
+#pragma unroll
+            for (int a = 0; a < NA; ++a) { b1[a] = INFINITY; b2[a] = INFINITY; bc[a] = cg; }
+            int chunk_id = cg;
+            for (int b = 0; b < n_btiles && ok; ++b, chunk_id += EW) {
+#pragma unroll
+                for (int a = 0; a < NA; ++a) {
+                    if (!ok) continue;
+                    const int slot = a % SLOTS;
+                    ok = mbar_wait(smem_u32(t_full + slot), (a / SLOTS) & 1, abort_flag);
+                    if (!ok) continue;
+                    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                    uint32_t v0[32], v1[32];
+                    TMEM_LD32(v0, tbase + slot * TN);
+                    TMEM_LD32(v1, tbase + slot * TN + 32);
+                    TMEM_WAIT32(v0);
+                    TMEM_WAIT32(v1);
+                    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0)
+                        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(t_empty + slot)) : "memory");
+                    const float m = chunk_min64(v0, v1);
+                    const bool better = m < b1[a];
+                    b2[a] = better ? b1[a] : fminf(b2[a], m);
+                    bc[a] = better ? chunk_id : bc[a];
+                    b1[a] = better ? m : b1[a];
+                }
+            }
+            // ---- merge the EW column groups of each point and store; the exchange area is reused by
+            //      the next group, hence the second barrier
+            if (cg > 0) {
+#pragma unroll
+                for (int a = 0; a < NA; ++a) {
+                    float* mrow = merge + (((cg - 1) * NA + a) * 3) * TM + r;
+                    mrow[0] = b1[a]; mrow[TM] = b2[a]; mrow[2 * TM] = __int_as_float(bc[a]);
+                }
+            }
+            asm volatile("bar.sync 1, %0;" ::"r"(EPI_WARPS * 32));
+            if (cg == 0 && ok && !*abort_flag) {
+                const int64_t base = ((int64_t)blockIdx.x + (int64_t)it * gridDim.x) * (NA * TM);
+#pragma unroll
+                for (int a = 0; a < NA; ++a) {
+                    const int64_t i = base + a * TM + r;
+                    if (i >= N) continue;
+                    float w1 = b1[a], w2 = b2[a];
+                    int wc = bc[a];
+#pragma unroll
+                    for (int o = 0; o < EW - 1; ++o) {
+                        const float* srow = merge + ((o * NA + a) * 3) * TM + r;
+                        const float o1 = srow[0], o2 = srow[TM];
+                        const int oc = __float_as_int(srow[2 * TM]);
+                        if (o1 < w1) { w2 = fminf(w1, o2); w1 = o1; wc = oc; }
+                        else { w2 = fminf(w2, o1); }
+                    }
+                    tstate[i] = make_float2(w2, __int_as_float(wc));
+                }
+            }
+            asm volatile("bar.sync 1, %0;" ::"r"(EPI_WARPS * 32));
+            ok = !*abort_flag;     // read after the barrier: the same answer in all sixteen warps
+        }
+    }
+    if (nonfinite) atomicOr(status, CC_DEV_NONFINITE);
     if (*abort_flag && lane == 0) atomicOr(status, CC_DEV_TIMEOUT);
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -677,7 +933,15 @@ cudaError_t launch_tensor(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int
             ProfScope ps(ctx, CC_K_ASSIGN_MAIN, st);
             // CTAs with a full set of NA point tiles, then the ragged rest
             const int64_t full_blocks = (na_per_cta == NA) ? n_tiles / NA : 0;
-            if (full_blocks > 0)
+            if (PersistCfg<G>::OK && full_blocks >= 2 * (int64_t)ctx->sm_count && full_blocks < (1ll << 30)) {
+                static bool attr_p = false;
+                if (!attr_p) {
+                    if ((e = cudaFuncSetAttribute(assign_tensor_persistent_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, PersistCfg<G>::SMEM)) != cudaSuccess) return e;
+                    attr_p = true;
+                }
+                assign_tensor_persistent_kernel<G><<<ctx->sm_count, PERSIST_THREADS, PersistCfg<G>::SMEM, st>>>(
+                    X, N, gB, Kpad / TN, (int)full_blocks, tstate, status);
+            } else if (full_blocks > 0)
                 assign_tensor_kernel<G, false, true><<<(unsigned)full_blocks, TC_THREADS, Cfg::SMEM, st>>>(
                     X, N, gB, Kpad / TN, NA, 0, params, tstate, status, nullptr, 0);
             const int64_t rest_tiles = n_tiles - full_blocks * NA;

@@ -132,6 +132,12 @@ cc_status cc_init_positions(int64_t N, int K, uint64_t seed, int64_t* positions_
 cc_status cc_init_codebook(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, int K, uint64_t seed,
                            float* C, void* stream);
 
+/* Caller-chosen initial codebook (for reproducing a run or starting from another method's centroids;
+ * the paper only uses its library's default start): copies K x g FP32 values from C0, which may be
+ * a host or a device pointer, to the device array C on `stream`.  A pageable host source is staged
+ * before the call returns; a pinned one must stay valid until the stream has passed the copy. */
+cc_status cc_set_codebook(cc_ctx* ctx, const float* C0_host_or_device, int K, int g, float* C, void* stream);
+
 /* E-step of Section 3.1: idx[i] = the centroid minimising ||x_i - c_j||^2 (lowest j on exact
  * ties), dist[i] = that squared distance (FP32), *objective = sum_i dist[i] (the Section 3.1
  * objective for this assignment, a plain sum).  X: N x g FP16; C: K x g FP32.

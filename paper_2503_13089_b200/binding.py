@@ -45,6 +45,7 @@ SIGNATURES = {
     "cc_reshape_subvectors": (_i32, [_vp, _vp, _i64, _i64, _i32, _i32, _vp, _vp]),
     "cc_init_positions": (_i32, [_i64, _i32, _u64, _vp]),
     "cc_init_codebook": (_i32, [_vp, _vp, _i64, _i32, _i32, _u64, _vp, _vp]),
+    "cc_set_codebook": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp]),
     "cc_assign": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp]),
     "cc_tensor_scores_ld": (_i64, [_i32]),
     "cc_tensor_scores": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp]),
@@ -197,6 +198,16 @@ def cc_init_positions(N: int, K: int, seed: int):
 
 def cc_init_codebook(ctx, X, N, g, K, seed, C, stream=None) -> None:
     _check(load().cc_init_codebook(ctx._h, _ptr(X), N, g, K, seed, _ptr(C), _stream(stream)), "cc_init_codebook")
+
+
+def cc_set_codebook(ctx, C0, K, g, C, stream=None) -> None:
+    """C0: a torch tensor on the host or on the device, or a contiguous float32 numpy array."""
+    if hasattr(C0, "ctypes"):
+        assert C0.dtype.name == "float32" and C0.flags["C_CONTIGUOUS"]
+        src = C0.ctypes.data
+    else:
+        src = _ptr(C0)
+    _check(load().cc_set_codebook(ctx._h, src, K, g, _ptr(C), _stream(stream)), "cc_set_codebook")
 
 
 def cc_assign(ctx, X, N, g, C, K, idx, dist=None, objective=None, n_resolved=None, stream=None) -> None:

@@ -237,6 +237,15 @@ cc_status cc_init_codebook(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, int
     return from_cuda(cc_launch_gather_init(ctx, X, g, K, pos_dev, C, st));
 }
 
+cc_status cc_set_codebook(cc_ctx* ctx, const float* C0, int K, int g, float* C, void* stream) {
+    if (!ctx || !C0 || !C) return CC_ERR_NULL;
+    if (g < 1 || g > 16) return CC_ERR_UNSUPPORTED_G;
+    if (K < 1 || K > 65536) return CC_ERR_K_RANGE;
+    if (!aligned16(C)) return CC_ERR_ALIGN;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    return from_cuda(cudaMemcpyAsync(C, C0, sizeof(float) * (size_t)K * g, cudaMemcpyDefault, (cudaStream_t)stream));
+}
+
 cc_status cc_assign(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const float* C, int K, uint16_t* idx,
                     float* dist, double* objective, int64_t* n_resolved, void* stream) {
     if (!ctx || !C || (N > 0 && (!X || !idx))) return CC_ERR_NULL;

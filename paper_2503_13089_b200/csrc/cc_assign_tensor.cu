@@ -793,7 +793,8 @@ assign_tensor_persistent_kernel(const uint16_t* __restrict__ X, int64_t N, const
 }
 
 // Finish, LPP = 8 lanes per point (four points per warp): lane k of a group recomputes the scores of
-// centroids 4k .. 4k+3 and 32+4k .. 32+4k+3 of the winning 64-centroid chunk with the FMA chain
+// centroids 4k .. 4k+3 and 32+4k .. 32+4k+3 (four consecutive centroids every 4 LPP) of the winning
+// 64-centroid chunk with the FMA chain
 // s = fma(x_{g-1}, m_{g-1}, ... fma(x_0, m_0, ||c||^2)), keeping its smallest score, its index and
 // its runner-up; a butterfly over the group gives every lane the chunk's winner and runner-up;
 // then the squared distance to the winner in FP64 (sub, mul, add in dimension order, no
@@ -826,7 +827,7 @@ finish_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __r
         float s1 = INFINITY, s2 = INFINITY;
         int j1 = 4 * k;
 #pragma unroll
-        for (int hf = 0; hf < 2; ++hf) {
+        for (int hf = 0; hf < TCHUNK / 4 / LPP; ++hf) {
             const float4 cs = __ldg(blk + G * (TCHUNK / 4) + hf * LPP);
             float s[4] = {cs.x, cs.y, cs.z, cs.w};
 #pragma unroll
@@ -841,7 +842,7 @@ finish_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __r
             for (int e = 0; e < 4; ++e) {
                 const bool take = s[e] < s1;                 // ascending index: strict '<' keeps the lowest
                 s2 = take ? s1 : fminf(s2, s[e]);
-                j1 = take ? hf * 32 + 4 * k + e : j1;
+                j1 = take ? (hf * LPP + k) * 4 + e : j1;
                 s1 = take ? s[e] : s1;
             }
         }

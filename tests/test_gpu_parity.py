@@ -338,6 +338,22 @@ def test_fit_moves_only_changed_points_yet_matches_the_driven_loop(N, g, K, iter
     assert np.array_equal(counts_or, counts)
 
 
+def test_set_codebook_from_host_and_device():
+    cc, u = _cc(), _u()
+    C0 = wl.make_codebook(333, 6, 3)
+    C = torch.zeros((333, 6), dtype=torch.float32, device="cuda")
+    cc.cc_set_codebook(u.ctx(), C0, 333, 6, C)                       # pageable host memory
+    torch.cuda.synchronize()
+    assert np.array_equal(C.cpu().numpy(), C0)
+    C2 = torch.zeros_like(C)
+    cc.cc_set_codebook(u.ctx(), C, 333, 6, C2)                       # device to device
+    torch.cuda.synchronize()
+    assert np.array_equal(C2.cpu().numpy(), C0)
+    with pytest.raises(cc.CCError) as e:
+        cc.cc_set_codebook(u.ctx(), C0, 70000, 6, C)
+    assert e.value.status == 4
+
+
 def test_blobs_recovered_and_k_equals_n():
     u = _u()
     X, labels, centres = wl.make_blobs(12, 300, 4, seed=90, sep=1.0, sigma=0.01)

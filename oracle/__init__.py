@@ -49,6 +49,7 @@ def _load():
         lib.oc_point_dist.restype = dbl
         lib.oc_point_dist.argtypes = [vp, i64, i32, vp, i32]
         lib.oc_update.argtypes = [vp, i64, i32, vp, i32, vp, vp]
+        lib.oc_codebook_grad.argtypes = [vp, i64, i32, vp, i32, vp]
         lib.oc_fit.argtypes = [vp, i64, i32, i32, i32, vp, vp, vp, vp, vp]
         lib.oc_float_to_half.argtypes = [vp, i64, vp]
         lib.oc_half_to_double.argtypes = [vp, i64, vp]
@@ -149,6 +150,17 @@ def update(X: np.ndarray, idx: np.ndarray, C_prev: np.ndarray) -> Tuple[np.ndarr
     counts = np.empty(K, dtype=np.int64)
     _load().oc_update(_p(X), N, g, _p(idx), K, _p(C), _p(counts))
     return C, counts
+
+
+def codebook_grad(dX: np.ndarray, idx: np.ndarray, K: int) -> np.ndarray:
+    """dC[j] = sum of dX[i] over the sub-vectors coded j (K x g float32)."""
+    dX = _half(dX)
+    N, g = dX.shape
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    assert idx.shape == (N,) and (N == 0 or (idx.min() >= 0 and idx.max() < K))
+    dC = np.empty((K, g), dtype=np.float32)
+    _load().oc_codebook_grad(_p(dX), N, g, _p(idx), K, _p(dC))
+    return dC
 
 
 def fit(X: np.ndarray, C0: np.ndarray, iters: int):

@@ -215,6 +215,21 @@ void oc_update(const uint16_t* X, int64_t N, int g, const int32_t* idx, int K, f
     free(sum);
 }
 
+/* ---- Gradient of the reconstruction with respect to the codebook ----------------
+ * The decoded weights are codebook[code] (appendix listing) and the paper trains only the
+ * codebook with the codes fixed (Sections 3.2-3.3), so by the chain rule the gradient of any
+ * loss with respect to centroid j is the sum of the gradients of the sub-vectors coded j:
+ * dC[j][t] = sum_{i : idx[i] = j} dX[i][t].  Double sums, one rounding to float. */
+void oc_codebook_grad(const uint16_t* dX, int64_t N, int g, const int32_t* idx, int K, float* dC) {
+    double* sum = (double*)calloc((size_t)K * g, sizeof(double));
+    for (int64_t i = 0; i < N; ++i) {
+        int32_t j = idx[i];
+        for (int t = 0; t < g; ++t) sum[(int64_t)j * g + t] += half_to_double(dX[i * g + t]);
+    }
+    for (int64_t e = 0; e < (int64_t)K * g; ++e) dC[e] = (float)sum[e];
+    free(sum);
+}
+
 /* ---- Lloyd loop: iters x (E-step, M-step); centroid state held in float -------- */
 /* objective[t] = sum_i d1_i at the t-th E-step (a plain sum, as in Section 3.1).  */
 void oc_fit(const uint16_t* X, int64_t N, int g, int K, int iters, float* C, int32_t* idx,

@@ -372,3 +372,40 @@ def test_workload_generators_are_seeded_and_shaped():
     assert np.isfinite(W1.astype(np.float32)).all()
     sel = wl.subset_positions(1000, 0.01, 3)
     assert len(sel) == 10 and len(set(sel.tolist())) == 10
+
+
+# ------------------------------------------------------------------ codebook gradient
+
+def test_codebook_grad_against_exact_rationals_autograd_and_the_m_step():
+    """dC[j] = sum of dX[i] over idx[i] = j: exact rational sums on a small case, torch autograd
+    of the gather codebook[code] in float64, linearity in dX, and counts x mean of the M-step."""
+    from fractions import Fraction
+    import torch
+    rng = np.random.default_rng(17)
+    N, g, K = 300, 5, 11
+    dX = (rng.standard_normal((N, g)) * rng.choice([1e-3, 1.0, 300.0], (N, 1))).astype(np.float16)
+    idx = rng.integers(0, K - 2, N).astype(np.int32)              # two clusters get no gradient
+    got = oracle.codebook_grad(dX, idx, K)
+    want = np.zeros((K, g), dtype=np.float32)
+    for j in range(K):
+        for t in range(g):
+            sacc = sum((Fraction(float(v)) for v in dX[idx == j, t]), Fraction(0))
+            want[j, t] = np.float32(float(sacc))                  # Fraction -> double -> float: sums fit a double here
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    assert np.all(got[K - 2:] == 0)
+    # autograd of the gather: loss = sum(codebook[code] * dX) has gradient index_add(dX)
+    Cb = torch.zeros((K, g), dtype=torch.float64, requires_grad=True)
+    (Cb[torch.from_numpy(idx.astype(np.int64))] * torch.from_numpy(dX.astype(np.float64))).sum().backward()
+    assert np.array_equal(got, Cb.grad.numpy().astype(np.float32))
+    # linearity where the sum of the two gradients is itself FP16-exact
+    a = (rng.integers(-8, 9, (N, g)) * 0.25).astype(np.float16)
+    b = (rng.integers(-8, 9, (N, g)) * 0.5).astype(np.float16)
+    assert np.array_equal(oracle.codebook_grad((a + b).astype(np.float16), idx, K),
+                          oracle.codebook_grad(a, idx, K) + oracle.codebook_grad(b, idx, K))
+    # the M-step's mean times its count is the same sum (values chosen so that every step is exact)
+    C_new, counts = oracle.update(a, idx, np.zeros((K, g), np.float32))
+    nz = counts > 0
+    assert np.allclose(oracle.codebook_grad(a, idx, K)[nz], C_new[nz] * counts[nz, None], rtol=1e-6, atol=0)
+    # K = 1: the column sums
+    assert np.array_equal(oracle.codebook_grad(a, np.zeros(N, np.int32), 1)[0],
+                          a.astype(np.float64).sum(0).astype(np.float32))

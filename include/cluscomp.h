@@ -195,6 +195,16 @@ cc_status cc_update(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const uint
 cc_status cc_update_static(int device, const uint16_t* X, int64_t N, int g, const uint16_t* idx, int K,
                            float* C, int32_t* counts, void* stream);
 
+/* Gradient with respect to the codebook (Sections 3.2-3.3: block-wise error minimisation, recovery
+ * training and finetuning all train the codebook with the codes kept fixed; the layer's weight is
+ * codebook[code], appendix listing).  By the chain rule dC[j] = sum over the sub-vectors coded j of
+ * dX[i], where dX is the gradient with respect to the decoded weight cut into sub-vectors exactly
+ * as cc_reshape_subvectors cuts W (padded coordinates are zero there and contribute nothing).
+ * dX: N x g FP16.  dC (out): K x g FP32, the exact integer sum rounded once; clusters without a
+ * member get 0.  Deterministic: the result does not depend on the order of the points. */
+cc_status cc_codebook_grad(cc_ctx* ctx, const uint16_t* dX, int64_t N, int g, const uint16_t* idx, int K,
+                           float* dC, void* stream);
+
 /* Lloyd loop of Section 3.1: iters x (E-step, M-step), no early stop (the paper runs a fixed
  * 20).  C: in = initial, out = after the last M-step.  idx / dist / counts (out): those of the
  * last iteration.  objective_trace (out, device, may be NULL): iters doubles, entry t = the

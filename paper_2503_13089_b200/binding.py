@@ -51,6 +51,7 @@ SIGNATURES = {
     "cc_tensor_scores": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp]),
     "cc_update": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp]),
     "cc_update_static": (_i32, [_i32, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp]),
+    "cc_codebook_grad": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp]),
     "cc_fit": (_i32, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "cc_finalize": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp]),
     "cc_decode": (_i32, [_vp, _vp, _i32, _i32, _vp, _i64, _i64, _i32, _vp, _vp]),
@@ -234,6 +235,11 @@ def cc_update_static(device, X, N, g, idx, K, C, counts, stream=None) -> None:
     accumulators are a fixed array inside the library (K * g <= UPDATE_STATIC_MAX_KG)."""
     _check(load().cc_update_static(device, _ptr(X), N, g, _ptr(idx), K, _ptr(C), _ptr(counts), _stream(stream)),
            "cc_update_static")
+
+
+def cc_codebook_grad(ctx, dX, N, g, idx, K, dC, stream=None) -> None:
+    _check(load().cc_codebook_grad(ctx._h, _ptr(dX), N, g, _ptr(idx), K, _ptr(dC), _stream(stream)),
+           "cc_codebook_grad")
 
 
 def cc_fit(ctx, X, N, g, K, iters, C, idx, dist, counts, objective_trace=None, stream=None) -> None:

@@ -282,6 +282,17 @@ cc_status cc_update(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const uint
     return from_cuda(cc_launch_update(ctx, L, X, N, g, idx, K, C, counts, (cudaStream_t)stream));
 }
 
+cc_status cc_codebook_grad(cc_ctx* ctx, const uint16_t* dX, int64_t N, int g, const uint16_t* idx, int K, float* dC,
+                           void* stream) {
+    if (!ctx || !dC || (N > 0 && (!dX || !idx))) return CC_ERR_NULL;
+    cc_status s = check_common(ctx, N, g, K, true);
+    if (s != CC_OK) return s;
+    if (!aligned16(dX) || !aligned16(dC)) return CC_ERR_ALIGN;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    const WsLayout L = cc_ws_layout(N, g, K);
+    return from_cuda(cc_launch_codebook_grad(ctx, L, dX, N, g, idx, K, dC, (cudaStream_t)stream));
+}
+
 cc_status cc_fit(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, int K, int iters, float* C, uint16_t* idx,
                  float* dist, int32_t* counts, double* objective_trace, void* stream) {
     if (!ctx || !X || !C || !idx || !counts) return CC_ERR_NULL;

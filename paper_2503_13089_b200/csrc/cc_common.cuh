@@ -106,5 +106,7 @@ cudaError_t cc_launch_assign_tail(cc_ctx*, const WsLayout&, const uint16_t* X, i
 
 cudaError_t cc_launch_update(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const uint16_t* idx,
                              int K, float* C, int32_t* counts, cudaStream_t);
+cudaError_t cc_launch_codebook_grad(cc_ctx*, const WsLayout&, const uint16_t* dX, int64_t N, int g, const uint16_t* idx,
+                                    int K, float* dC, cudaStream_t);
 cudaError_t cc_launch_update_delta(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const uint16_t* idx,
                                    uint16_t* idx_prev, int K, float* C, int32_t* counts, cudaStream_t);

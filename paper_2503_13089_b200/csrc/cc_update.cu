@@ -106,6 +106,15 @@ update_finish_kernel(const long long* __restrict__ sum_lo, const long long* __re
     C[e] = (float)(s / (double)n);
 }
 
+// Gradient with respect to the codebook: the exact integer sums as they are, rounded once to FP32.
+__global__ void __launch_bounds__(256)
+grad_finish_kernel(const long long* __restrict__ sum_lo, const long long* __restrict__ sum_hi, int n,
+                   float* __restrict__ dC) {
+    const int e = blockIdx.x * blockDim.x + threadIdx.x;
+    if (e >= n) return;
+    dC[e] = (float)((double)sum_lo[e] * 5.9604644775390625e-8 + (double)sum_hi[e] * 0.0078125);
+}
+
 }  // namespace
 
 #define CC_UPDATE_DISPATCH(g, CALL)                                                                           \
@@ -150,6 +159,29 @@ cudaError_t cc_launch_update(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, 
     ProfScope ps(ctx, CC_K_UPDATE_FINISH, st);
     update_finish_kernel<<<(K * g + 255) / 256, 256, 0, st>>>(reinterpret_cast<long long*>(sum_lo),
                                                              reinterpret_cast<long long*>(sum_hi), counts, K, g, C);
+    return cudaGetLastError();
+}
+
+// dC[j] = sum of dX[i] over idx[i] = j, with the M-step's exact accumulation (scratch counts in the
+// workspace: the position list of the initialisation is free by then).
+cudaError_t cc_launch_codebook_grad(cc_ctx* ctx, const WsLayout& L, const uint16_t* dX, int64_t N, int g,
+                                    const uint16_t* idx, int K, float* dC, cudaStream_t st) {
+    char* ws = static_cast<char*>(ctx->ws);
+    ull* sum_lo = reinterpret_cast<ull*>(ws + L.sum_lo);
+    ull* sum_hi = reinterpret_cast<ull*>(ws + L.sum_hi);
+    int32_t* counts = reinterpret_cast<int32_t*>(ws + L.positions);
+    cudaError_t e;
+    if ((e = cudaMemsetAsync(sum_lo, 0, L.tmp_c - L.sum_lo, st)) != cudaSuccess) return e;
+    if ((e = cudaMemsetAsync(counts, 0, sizeof(int32_t) * (size_t)K, st)) != cudaSuccess) return e;
+    if (N > 0) {
+#define CALL(G) e = launch_accumulate<G>(ctx, dX, N, idx, K, sum_lo, sum_hi, counts, st)
+        CC_UPDATE_DISPATCH(g, CALL)
+#undef CALL
+        if (e != cudaSuccess) return e;
+    }
+    ProfScope ps(ctx, CC_K_UPDATE_FINISH, st);
+    grad_finish_kernel<<<(K * g + 255) / 256, 256, 0, st>>>(reinterpret_cast<long long*>(sum_lo),
+                                                            reinterpret_cast<long long*>(sum_hi), K * g, dC);
     return cudaGetLastError();
 }
 

@@ -256,6 +256,30 @@ def test_update_large_and_tiny_values_and_point_order():
     assert np.array_equal(C_perm.view(np.uint32), C_gpu.view(np.uint32))
 
 
+@pytest.mark.parametrize("N,g,K", [(1, 4, 3), (70001, 4, 1000), (9000, 8, 5000), (6000, 16, 129), (3001, 9, 200),
+                                   (200000, 6, 65500)])
+def test_codebook_grad_matches_oracle_bit_for_bit(N, g, K):
+    """Gradient of the decoded weights pushed back to the codebook: exact integer sums on the GPU,
+    float64 sums in the oracle, both rounded once, so the bits must agree; empty clusters get 0."""
+    cc, u = _cc(), _u()
+    rng = np.random.default_rng(N + K)
+    dX = (rng.standard_normal((N, g)) * rng.choice([1e-4, 0.05, 40.0], (N, 1))).astype(np.float16)
+    idx = rng.integers(0, max(1, K - 2), N).astype(np.int32)
+    want = oracle.codebook_grad(dX, idx, K)
+    c = u.ctx()
+    c.ensure_workspace(N, g, K)
+    dC = torch.full((K, g), 7.0, dtype=torch.float32, device="cuda")
+    idxd = torch.from_numpy(idx.astype(np.uint16).view(np.int16)).cuda().view(torch.uint16)
+    cc.cc_codebook_grad(c, u.half_dev(dX), N, g, idxd, K, dC)
+    cc.cc_poll_status(c)
+    got = dC.cpu().numpy()
+    assert np.array_equal(got.view(np.uint32), want.view(np.uint32))
+    p = rng.permutation(N)                                   # order of the sub-vectors must not matter
+    idxp = torch.from_numpy(idx[p].astype(np.uint16).view(np.int16)).cuda().view(torch.uint16)
+    cc.cc_codebook_grad(c, u.half_dev(dX[p]), N, g, idxp, K, dC)
+    assert np.array_equal(dC.cpu().numpy().view(np.uint32), want.view(np.uint32))
+
+
 # ------------------------------------------------------------------ Lloyd loop
 
 def _lockstep(X, C0, iters, full_oracle=True, sel=None):

@@ -385,28 +385,35 @@ __device__ __forceinline__ double block_sum(double v, double* sh) {
     return r;   // valid in thread 0
 }
 
+// One kernel: every block writes the FP64 sum of its slice of dist; the block that finishes last
+// (a ticket in status word 8, left at zero again) adds the partial sums in a fixed order, so the
+// result does not depend on which block that is.
 __global__ void __launch_bounds__(256)
-objective_partial_kernel(const float* __restrict__ dist, int64_t N, double* __restrict__ partials) {
+objective_kernel(const float* __restrict__ dist, int64_t N, double* __restrict__ partials, unsigned* __restrict__ status,
+                 double* __restrict__ objective, int64_t* __restrict__ n_resolved) {
     __shared__ double sh[8];
+    __shared__ bool last;
     const int64_t per = (N + gridDim.x - 1) / gridDim.x;
     const int64_t lo = (int64_t)blockIdx.x * per;
     const int64_t hi = (lo + per < N) ? lo + per : N;
     double acc = 0.0;
     for (int64_t i = lo + threadIdx.x; i < hi; i += blockDim.x) acc += (double)dist[i];
     const double r = block_sum(acc, sh);
-    if (threadIdx.x == 0) partials[blockIdx.x] = r;
-}
-
-__global__ void __launch_bounds__(256)
-objective_final_kernel(const double* __restrict__ partials, int n, const unsigned* __restrict__ status,
-                       double* __restrict__ objective, int64_t* __restrict__ n_resolved) {
-    __shared__ double sh[8];
-    double acc = 0.0;
-    for (int i = threadIdx.x; i < n; i += blockDim.x) acc += partials[i];
-    const double r = block_sum(acc, sh);
     if (threadIdx.x == 0) {
-        if (objective) *objective = r;
+        partials[blockIdx.x] = r;
+        __threadfence();
+        last = atomicAdd(status + 8, 1u) == gridDim.x - 1;
+    }
+    __syncthreads();
+    if (!last) return;
+    __threadfence();
+    double tot = 0.0;
+    for (int i = threadIdx.x; i < (int)gridDim.x; i += blockDim.x) tot += __ldcg(partials + i);
+    const double t = block_sum(tot, sh);
+    if (threadIdx.x == 0) {
+        if (objective) *objective = t;
         if (n_resolved) *n_resolved = (int64_t)*reinterpret_cast<const ull*>(status + 2);
+        status[8] = 0u;
     }
 }
 
@@ -454,12 +461,9 @@ cudaError_t launch_tail(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64
     if (objective || n_resolved) {
         int blocks = (int)((N + 4095) / 4096);
         if (blocks > CC_OBJ_BLOCKS) blocks = CC_OBJ_BLOCKS;
-        if (blocks > 0) {
-            ProfScope ps(ctx, CC_K_OBJECTIVE, st);
-            objective_partial_kernel<<<blocks, 256, 0, st>>>(dist, N, partials);
-        }
+        if (blocks < 1) blocks = 1;
         ProfScope ps(ctx, CC_K_OBJECTIVE, st);
-        objective_final_kernel<<<1, 256, 0, st>>>(partials, blocks, status, objective, n_resolved);
+        objective_kernel<<<blocks, 256, 0, st>>>(dist, N, partials, status, objective, n_resolved);
     }
     return cudaGetLastError();
 }

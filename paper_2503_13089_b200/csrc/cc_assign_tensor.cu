@@ -170,7 +170,7 @@ __device__ __forceinline__ float qconst(int p) {   // 2^15, 2^6, 2^-3, 2^-12
 template <int G>
 __global__ void __launch_bounds__(256)
 prep_tensor_kernel(const float* __restrict__ C, int K, int Kpad, TcParams* __restrict__ params,
-                   uint16_t* __restrict__ gB) {
+                   uint16_t* __restrict__ gB, float* __restrict__ rescan) {
     using Cfg = TcCfg<G>;
     constexpr int KD = Cfg::KD, SPLIT = Cfg::SPLIT;
     const float S = scale_from_range(params->cmax_bits, params->qmax_bits);
@@ -178,6 +178,20 @@ prep_tensor_kernel(const float* __restrict__ C, int K, int Kpad, TcParams* __res
     if (e == 0) { params->S = S; params->invS = 1.0f / S; }
     if (e >= Kpad * (KD / 8)) return;
     const int j = e / (KD / 8), kc = e - j * (KD / 8);
+    if (kc == 0 && rescan) {
+        // FP32 table of the finish kernel, one block of (g+1) x 64 floats per 64-centroid chunk: for
+        // coordinate t the 64 values m_{j,t} = -2 c_{j,t} of the chunk side by side, then the 64 squared
+        // norms (a group of 8 lanes reads 128 contiguous bytes per load); padding can never win
+        float* blk = rescan + (int64_t)(j / TCHUNK) * ((G + 1) * TCHUNK) + (j % TCHUNK);
+        double s = 0.0;
+#pragma unroll
+        for (int t = 0; t < G; ++t) {
+            const float c = (j < K) ? C[(int64_t)j * G + t] : 0.f;
+            blk[t * TCHUNK] = -2.0f * c;
+            s += (double)c * (double)c;
+        }
+        blk[G * TCHUNK] = (j < K) ? (float)s : kBig;
+    }
     __half out[8];
     __half qp[NQ];
     bool need_q = false;
@@ -231,26 +245,6 @@ prep_tensor_kernel(const float* __restrict__ C, int K, int Kpad, TcParams* __res
     w.z = (unsigned)__half_as_ushort(out[4]) | ((unsigned)__half_as_ushort(out[5]) << 16);
     w.w = (unsigned)__half_as_ushort(out[6]) | ((unsigned)__half_as_ushort(out[7]) << 16);
     *reinterpret_cast<uint4*>(dst) = w;
-}
-
-// FP32 codebook of the finish kernel, one block of (g+1) x 64 floats per 64-centroid chunk: for
-// coordinate t the 64 values m_{j,t} = -2 c_{j,t} of the chunk's centroids side by side, then their
-// 64 squared norms.  A group of 8 lanes reads 128 contiguous bytes per load.  Centroids
-// K .. Kpad-1 are padding that can never win.
-template <int G>
-__global__ void __launch_bounds__(256)
-prep_rescan_kernel(const float* __restrict__ C, int K, int Kpad, float* __restrict__ rescan) {
-    const int j = blockIdx.x * blockDim.x + threadIdx.x;
-    if (j >= Kpad) return;
-    float* blk = rescan + (int64_t)(j / TCHUNK) * ((G + 1) * TCHUNK) + (j % TCHUNK);
-    double s = 0.0;
-#pragma unroll
-    for (int t = 0; t < G; ++t) {
-        const float c = (j < K) ? C[(int64_t)j * G + t] : 0.f;
-        blk[t * TCHUNK] = -2.0f * c;
-        s += (double)c * (double)c;
-    }
-    blk[G * TCHUNK] = (j < K) ? (float)s : kBig;
 }
 
 #define TMEM_LD32(v, taddr)                                                                                      \
@@ -896,9 +890,9 @@ cudaError_t launch_tensor(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int
     // FP32 rows of the finish kernel sit behind the FP16 operand image (at most 96 bytes per centroid)
     float* rescan = reinterpret_cast<float*>(ws + L.tensor + (size_t)Kpad * 96);
     cudaError_t e;
-    // status words 2..3 (the flagged-point counter of this E-step) and the range words
-    if ((e = cudaMemsetAsync(status + 2, 0, 8, st)) != cudaSuccess) return e;
-    if ((e = cudaMemsetAsync(params, 0, sizeof(TcParams), st)) != cudaSuccess) return e;
+    // status words 2..3 (the flagged-point counter of this E-step) up to the range words: one memset
+    // (the words in between are unused except the objective's ticket, which is zero between kernels)
+    if ((e = cudaMemsetAsync(status + 2, 0, 120 + sizeof(TcParams), st)) != cudaSuccess) return e;
     {
         ProfScope ps(ctx, CC_K_ASSIGN_PREP, st);
         tensor_range_kernel<<<(K + 255) / 256, 256, 0, st>>>(C, K, G, params);
@@ -906,11 +900,7 @@ cudaError_t launch_tensor(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int
     {
         ProfScope ps(ctx, CC_K_ASSIGN_PREP, st);
         const int n = Kpad * (Cfg::KD / 8);
-        prep_tensor_kernel<G><<<(n + 255) / 256, 256, 0, st>>>(C, K, Kpad, params, gB);
-    }
-    if (!dump) {
-        ProfScope ps(ctx, CC_K_ASSIGN_PREP, st);
-        prep_rescan_kernel<G><<<(Kpad + 255) / 256, 256, 0, st>>>(C, K, Kpad, rescan);
+        prep_tensor_kernel<G><<<(n + 255) / 256, 256, 0, st>>>(C, K, Kpad, params, gB, dump ? nullptr : rescan);
     }
     if (N > 0) {
         const int64_t n_tiles = (N + TM - 1) / TM;

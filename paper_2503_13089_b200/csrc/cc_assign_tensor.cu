@@ -906,7 +906,9 @@ cudaError_t launch_tensor(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int
         const int64_t n_tiles = (N + TM - 1) / TM;
         int64_t na_per_cta = (n_tiles + ctx->sm_count - 1) / ctx->sm_count;    // small inputs still use every SM
         if (na_per_cta > NA) na_per_cta = NA;
-        static bool attr_set = false;
+        // the opt-in to large dynamic shared memory is per device
+        static bool attr_set_dev[64] = {};
+        bool& attr_set = attr_set_dev[ctx->device & 63];
         if (!attr_set) {
             if ((e = cudaFuncSetAttribute(assign_tensor_kernel<G, true, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM)) != cudaSuccess) return e;
             if ((e = cudaFuncSetAttribute(assign_tensor_kernel<G, false, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM)) != cudaSuccess) return e;
@@ -925,7 +927,8 @@ cudaError_t launch_tensor(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int
             // CTAs with a full set of NA point tiles, then the ragged rest
             const int64_t full_blocks = (na_per_cta == NA) ? n_tiles / NA : 0;
             if (PersistCfg<G>::OK && full_blocks >= 2 * (int64_t)ctx->sm_count && full_blocks < (1ll << 30)) {
-                static bool attr_p = false;
+                static bool attr_p_dev[64] = {};
+                bool& attr_p = attr_p_dev[ctx->device & 63];
                 if (!attr_p) {
                     if ((e = cudaFuncSetAttribute(assign_tensor_persistent_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, PersistCfg<G>::SMEM)) != cudaSuccess) return e;
                     attr_p = true;

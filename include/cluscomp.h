@@ -61,7 +61,7 @@ typedef enum {
                                in_features zero-padded to a multiple of g.                   */
 
 /* Which E-step kernel family cc_assign uses. */
-#define CC_PATH_AUTO 0   /* chosen per (g, K) from measurements                        */
+#define CC_PATH_AUTO 0   /* the faster path: measured, the tensor-core one for every g */
 #define CC_PATH_FFMA 1   /* FP32 FMA pipes, register-tiled                             */
 #define CC_PATH_TENSOR 2 /* tcgen05 tensor cores with TMEM accumulators                */
 

@@ -64,3 +64,17 @@ def test_no_gpu_fails_loudly():
     with pytest.raises(cc.CCError) as e:
         cc.Context(0)
     assert e.value.status == 10
+
+
+def test_workload_sizes_follow_the_padding_rule():
+    """Every shipped workload's sub-vector count is the listing's padded num_codes, as the library and the
+    oracle compute it (the paper-grid workloads have out_features that g does not divide)."""
+    from paper_2503_13089_b200 import workloads as wl
+    padded = 0
+    for w in wl.WORKLOADS.values():
+        for m in w.matrices:
+            n = w.n_subvectors(m)
+            assert n == cc.cc_num_subvectors(m.d_out, m.d_in, w.g, 0) == oracle.num_subvectors(m.d_out, m.d_in, w.g, 0)
+            assert 1 <= w.K <= 65536 and n >= w.K
+            padded += m.d_out % w.g != 0
+    assert padded >= 4

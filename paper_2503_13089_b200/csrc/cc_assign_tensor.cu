@@ -29,6 +29,10 @@
 // smallest and second-smallest 64-centroid chunk minimum and the id of the best chunk (one
 // 3-input min per two scores); the index inside the chunk, the distance and the near-tie flag are
 // computed afterwards by the finish kernel from FP32 data.  Nothing N x K is written to memory.
+// Three instantiations share this structure: a persistent kernel (g <= 9: one CTA per SM walks over
+// groups of NA point tiles while an extra warp builds the next group's A operand), a one-group-per-
+// CTA kernel specialised for full groups (g >= 10), and a generic one for the ragged rest and for
+// small inputs.
 //
 // Every wait on an mbarrier is bounded (clock based); on a time-out the CTA raises the status
 // bit CC_DEV_TIMEOUT, stops issuing work, and still releases its tensor memory.

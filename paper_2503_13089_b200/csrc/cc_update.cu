@@ -8,6 +8,9 @@
 // arrive: the kernel is deterministic without sorting the points first, the counts are exact
 // integers, and the mean is rounded exactly once (sum -> double -> divide -> FP32).
 // A cluster with no member keeps its previous centroid.
+// The same property lets the Lloyd loop keep the sums between iterations and only move the points
+// whose code changed (update_delta_kernel), and gives the gradient with respect to the codebook
+// (the same sums without the division).
 #include "cc_common.cuh"
 
 namespace {

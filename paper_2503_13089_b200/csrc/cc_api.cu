@@ -16,8 +16,10 @@ WsLayout cc_ws_layout(int64_t N, int g, int K) {
     L.cprep = take(Kpad / 2 * (size_t)(g + 1) * 16);
     L.flagged = take((size_t)N * 4);
     L.partials = take((size_t)CC_OBJ_BLOCKS * 8);
-    L.sum_lo = take((size_t)K * g * 8);
-    L.sum_hi = take((size_t)K * g * 8);
+    const size_t R = (size_t)cc_sum_copies(K, g);
+    L.sum_lo = take(R * K * g * 8);
+    L.sum_hi = take(R * K * g * 8);
+    L.count_copies = take(R * K * 4);
     L.tmp_c = take((size_t)K * g * 4);
     L.positions = take((size_t)K * 8);
     L.dist_tmp = take((size_t)N * 4);

@@ -59,8 +59,9 @@ struct WsLayout {
     size_t cprep;      // staged codebook for the FFMA E-step
     size_t flagged;    // u32 list of points sent to the exact stage
     size_t partials;   // doubles: per-block objective partial sums
-    size_t sum_lo;     // int64 K x g: sums of |x| < 8 in units of 2^-24
-    size_t sum_hi;     // int64 K x g: sums of |x| >= 8 in units of 2^-7
+    size_t sum_lo;     // int64 R x K x g: sums of |x| < 8 in units of 2^-24 (R = cc_sum_copies)
+    size_t sum_hi;     // int64 R x K x g: sums of |x| >= 8 in units of 2^-7
+    size_t count_copies;  // int32 R x K: per-copy member counts of the M-step (R > 1)
     size_t tmp_c;      // float K x g: widened FP16 codebook (finalize)
     size_t positions;  // int64 K: initial positions
     size_t dist_tmp;   // float N: distances when the caller passes dist == NULL
@@ -74,6 +75,16 @@ constexpr int CC_KPAD = 1024;          // staged codebook is padded to a multipl
 constexpr int CC_OBJ_BLOCKS = 1024;    // partial sums of the objective reduction
 
 WsLayout cc_ws_layout(int64_t N, int g, int K);
+
+// Copies of the M-step's sums (small codebooks only: at most CC_SUM_COPY_ELEMS words per array).
+#ifndef CC_SUM_COPIES_MAX
+#define CC_SUM_COPIES_MAX 16
+#endif
+constexpr int CC_SUM_COPY_ELEMS = 262144;
+static inline int cc_sum_copies(int K, int g) {
+    const int r = CC_SUM_COPY_ELEMS / (K * g);
+    return r < 1 ? 1 : (r > CC_SUM_COPIES_MAX ? CC_SUM_COPIES_MAX : r);
+}
 
 static inline size_t cc_align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 

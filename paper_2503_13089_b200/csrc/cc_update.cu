@@ -30,36 +30,27 @@ __device__ __forceinline__ void add_coord(uint16_t h, ull* lo, ull* hi) {
     }
 }
 
+// One lane per coordinate: the G reductions of a point go to G adjacent 64-bit words (one 32-byte
+// sector at G = 4, one 128-byte line at G = 16), so a warp's reduction instruction touches 32 / G
+// sectors instead of 32.  With few clusters the same words are hit by many points at once and the
+// reductions queue up in L2; the sums are then kept in R copies (copy = block % R, one after the
+// other, `copy_elems` words apart; the counts likewise, K apart) which the finish kernel adds up.
 template <int G>
 __global__ void __launch_bounds__(256)
 update_accumulate_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* __restrict__ idx, int K,
-                         ull* __restrict__ sum_lo, ull* __restrict__ sum_hi, int* __restrict__ counts) {
-    for (int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; i < N; i += (int64_t)gridDim.x * blockDim.x) {
+                         ull* __restrict__ sum_lo, ull* __restrict__ sum_hi, int* __restrict__ counts, int R) {
+    const int copy = (int)(blockIdx.x % (unsigned)R);
+    sum_lo += (int64_t)copy * K * G;
+    sum_hi += (int64_t)copy * K * G;
+    counts += (int64_t)copy * K;
+    const int64_t total = N * G;
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
+        const int64_t i = e / G;
+        const int t = (int)(e - i * G);
         const int j = idx[i];
         if (j >= K) continue;
-        atomicAdd(counts + j, 1);
-        const uint16_t* row = X + i * G;
-        uint16_t h[G];
-        if constexpr (G % 8 == 0) {
-#pragma unroll
-            for (int v = 0; v < G / 8; ++v) {
-                uint4 u = __ldg(reinterpret_cast<const uint4*>(row) + v);
-                unsigned w[4] = {u.x, u.y, u.z, u.w};
-#pragma unroll
-                for (int k = 0; k < 4; ++k) { h[v * 8 + 2 * k] = w[k] & 0xffffu; h[v * 8 + 2 * k + 1] = w[k] >> 16; }
-            }
-        } else if constexpr (G % 4 == 0) {
-#pragma unroll
-            for (int v = 0; v < G / 4; ++v) {
-                uint2 u = __ldg(reinterpret_cast<const uint2*>(row) + v);
-                h[v * 4] = u.x & 0xffffu; h[v * 4 + 1] = u.x >> 16; h[v * 4 + 2] = u.y & 0xffffu; h[v * 4 + 3] = u.y >> 16;
-            }
-        } else {
-#pragma unroll
-            for (int t = 0; t < G; ++t) h[t] = __ldg(row + t);
-        }
-#pragma unroll
-        for (int t = 0; t < G; ++t) add_coord(h[t], sum_lo + (int64_t)j * G + t, sum_hi + (int64_t)j * G + t);
+        if (t == 0) atomicAdd(counts + j, 1);
+        add_coord(__ldg(X + e), sum_lo + (int64_t)j * G + t, sum_hi + (int64_t)j * G + t);
     }
 }
 
@@ -98,24 +89,45 @@ update_delta_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* _
     }
 }
 
+// Adds up the R copies of the sums and counts, leaves the totals in copy 0 and in `counts` (the
+// incremental M-step continues from those), and writes the means.  With R = 1, count_copies is
+// `counts` itself.
 __global__ void __launch_bounds__(256)
-update_finish_kernel(const long long* __restrict__ sum_lo, const long long* __restrict__ sum_hi,
-                     const int* __restrict__ counts, int K, int g, float* __restrict__ C) {
+update_finish_kernel(long long* __restrict__ sum_lo, long long* __restrict__ sum_hi, const int* count_copies,
+                     int* counts, int K, int g, int R, float* __restrict__ C) {
     const int e = blockIdx.x * blockDim.x + threadIdx.x;
-    if (e >= K * g) return;
-    const int n = counts[e / g];
+    const int KG = K * g;
+    if (e >= KG) return;
+    const int j = e / g;
+    long long lo = sum_lo[e], hi = sum_hi[e];
+    int n = count_copies[j];
+    if (R > 1) {
+        for (int r = 1; r < R; ++r) {
+            lo += sum_lo[(int64_t)r * KG + e];
+            hi += sum_hi[(int64_t)r * KG + e];
+            n += count_copies[(int64_t)r * K + j];
+        }
+        sum_lo[e] = lo;
+        sum_hi[e] = hi;
+        if (e == j * g) counts[j] = n;
+    }
     if (n <= 0) return;   // empty cluster: previous centroid stays
-    const double s = (double)sum_lo[e] * 5.9604644775390625e-8 + (double)sum_hi[e] * 0.0078125;
+    const double s = (double)lo * 5.9604644775390625e-8 + (double)hi * 0.0078125;
     C[e] = (float)(s / (double)n);
 }
 
 // Gradient with respect to the codebook: the exact integer sums as they are, rounded once to FP32.
 __global__ void __launch_bounds__(256)
-grad_finish_kernel(const long long* __restrict__ sum_lo, const long long* __restrict__ sum_hi, int n,
+grad_finish_kernel(const long long* __restrict__ sum_lo, const long long* __restrict__ sum_hi, int n, int R,
                    float* __restrict__ dC) {
     const int e = blockIdx.x * blockDim.x + threadIdx.x;
     if (e >= n) return;
-    dC[e] = (float)((double)sum_lo[e] * 5.9604644775390625e-8 + (double)sum_hi[e] * 0.0078125);
+    long long lo = 0, hi = 0;
+    for (int r = 0; r < R; ++r) {
+        lo += sum_lo[(int64_t)r * n + e];
+        hi += sum_hi[(int64_t)r * n + e];
+    }
+    dC[e] = (float)((double)lo * 5.9604644775390625e-8 + (double)hi * 0.0078125);
 }
 
 }  // namespace
@@ -132,14 +144,36 @@ grad_finish_kernel(const long long* __restrict__ sum_lo, const long long* __rest
 namespace {
 
 template <int G>
-cudaError_t launch_accumulate(cc_ctx* ctx, const uint16_t* X, int64_t N, const uint16_t* idx, int K, ull* sum_lo,
-                              ull* sum_hi, int32_t* counts, cudaStream_t st) {
-    ProfScope ps(ctx, CC_K_UPDATE_ACCUM, st);
-    int64_t blocks = (N + 255) / 256;
-    const int64_t cap = (int64_t)ctx->sm_count * 16;
+cudaError_t launch_accumulate(int sm_count, const uint16_t* X, int64_t N, const uint16_t* idx, int K, ull* sum_lo,
+                              ull* sum_hi, int32_t* counts, int R, cudaStream_t st) {
+    int64_t blocks = (N * G + 255) / 256;
+    const int64_t cap = (int64_t)sm_count * 16;
     if (blocks > cap) blocks = cap;
-    update_accumulate_kernel<G><<<(unsigned)blocks, 256, 0, st>>>(X, N, idx, K, sum_lo, sum_hi, counts);
+    update_accumulate_kernel<G><<<(unsigned)blocks, 256, 0, st>>>(X, N, idx, K, sum_lo, sum_hi, counts, R);
     return cudaGetLastError();
+}
+
+// Clears the R copies of the sums and counts and accumulates all points.  *count_copies is where
+// the (copies of the) counts were accumulated: the caller's array when R = 1.
+cudaError_t accumulate_all(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64_t N, int g, const uint16_t* idx,
+                           int K, int32_t* counts, int R, int32_t** count_copies, cudaStream_t st) {
+    char* ws = static_cast<char*>(ctx->ws);
+    ull* sum_lo = reinterpret_cast<ull*>(ws + L.sum_lo);
+    ull* sum_hi = reinterpret_cast<ull*>(ws + L.sum_hi);
+    int32_t* cc = R > 1 ? reinterpret_cast<int32_t*>(ws + L.count_copies) : counts;
+    *count_copies = cc;
+    const size_t used = sizeof(ull) * (size_t)K * g * R;
+    cudaError_t e;
+    if ((e = cudaMemsetAsync(sum_lo, 0, used, st)) != cudaSuccess) return e;
+    if ((e = cudaMemsetAsync(sum_hi, 0, used, st)) != cudaSuccess) return e;
+    if ((e = cudaMemsetAsync(cc, 0, sizeof(int32_t) * (size_t)K * R, st)) != cudaSuccess) return e;
+    if (N > 0) {
+        ProfScope ps(ctx, CC_K_UPDATE_ACCUM, st);
+#define CALL(G) e = launch_accumulate<G>(ctx->sm_count, X, N, idx, K, sum_lo, sum_hi, cc, R, st)
+        CC_UPDATE_DISPATCH(g, CALL)
+#undef CALL
+    }
+    return e;
 }
 
 }  // namespace
@@ -147,21 +181,14 @@ cudaError_t launch_accumulate(cc_ctx* ctx, const uint16_t* X, int64_t N, const u
 cudaError_t cc_launch_update(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64_t N, int g, const uint16_t* idx,
                              int K, float* C, int32_t* counts, cudaStream_t st) {
     char* ws = static_cast<char*>(ctx->ws);
-    ull* sum_lo = reinterpret_cast<ull*>(ws + L.sum_lo);
-    ull* sum_hi = reinterpret_cast<ull*>(ws + L.sum_hi);
-    cudaError_t e;
-    // sum_lo and sum_hi are adjacent in the workspace
-    if ((e = cudaMemsetAsync(sum_lo, 0, L.tmp_c - L.sum_lo, st)) != cudaSuccess) return e;
-    if ((e = cudaMemsetAsync(counts, 0, sizeof(int32_t) * (size_t)K, st)) != cudaSuccess) return e;
-    if (N > 0) {
-#define CALL(G) e = launch_accumulate<G>(ctx, X, N, idx, K, sum_lo, sum_hi, counts, st)
-        CC_UPDATE_DISPATCH(g, CALL)
-#undef CALL
-        if (e != cudaSuccess) return e;
-    }
+    const int R = cc_sum_copies(K, g);
+    int32_t* count_copies = nullptr;
+    const cudaError_t e = accumulate_all(ctx, L, X, N, g, idx, K, counts, R, &count_copies, st);
+    if (e != cudaSuccess) return e;
     ProfScope ps(ctx, CC_K_UPDATE_FINISH, st);
-    update_finish_kernel<<<(K * g + 255) / 256, 256, 0, st>>>(reinterpret_cast<long long*>(sum_lo),
-                                                             reinterpret_cast<long long*>(sum_hi), counts, K, g, C);
+    update_finish_kernel<<<(K * g + 255) / 256, 256, 0, st>>>(reinterpret_cast<long long*>(ws + L.sum_lo),
+                                                             reinterpret_cast<long long*>(ws + L.sum_hi),
+                                                             count_copies, counts, K, g, R, C);
     return cudaGetLastError();
 }
 
@@ -170,21 +197,14 @@ cudaError_t cc_launch_update(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, 
 cudaError_t cc_launch_codebook_grad(cc_ctx* ctx, const WsLayout& L, const uint16_t* dX, int64_t N, int g,
                                     const uint16_t* idx, int K, float* dC, cudaStream_t st) {
     char* ws = static_cast<char*>(ctx->ws);
-    ull* sum_lo = reinterpret_cast<ull*>(ws + L.sum_lo);
-    ull* sum_hi = reinterpret_cast<ull*>(ws + L.sum_hi);
     int32_t* counts = reinterpret_cast<int32_t*>(ws + L.positions);
-    cudaError_t e;
-    if ((e = cudaMemsetAsync(sum_lo, 0, L.tmp_c - L.sum_lo, st)) != cudaSuccess) return e;
-    if ((e = cudaMemsetAsync(counts, 0, sizeof(int32_t) * (size_t)K, st)) != cudaSuccess) return e;
-    if (N > 0) {
-#define CALL(G) e = launch_accumulate<G>(ctx, dX, N, idx, K, sum_lo, sum_hi, counts, st)
-        CC_UPDATE_DISPATCH(g, CALL)
-#undef CALL
-        if (e != cudaSuccess) return e;
-    }
+    const int R = cc_sum_copies(K, g);
+    int32_t* count_copies = nullptr;
+    const cudaError_t e = accumulate_all(ctx, L, dX, N, g, idx, K, counts, R, &count_copies, st);
+    if (e != cudaSuccess) return e;
     ProfScope ps(ctx, CC_K_UPDATE_FINISH, st);
-    grad_finish_kernel<<<(K * g + 255) / 256, 256, 0, st>>>(reinterpret_cast<long long*>(sum_lo),
-                                                            reinterpret_cast<long long*>(sum_hi), K * g, dC);
+    grad_finish_kernel<<<(K * g + 255) / 256, 256, 0, st>>>(reinterpret_cast<long long*>(ws + L.sum_lo),
+                                                           reinterpret_cast<long long*>(ws + L.sum_hi), K * g, R, dC);
     return cudaGetLastError();
 }
 
@@ -207,7 +227,8 @@ cudaError_t cc_launch_update_delta(cc_ctx* ctx, const WsLayout& L, const uint16_
     }
     ProfScope ps(ctx, CC_K_UPDATE_FINISH, st);
     update_finish_kernel<<<(K * g + 255) / 256, 256, 0, st>>>(reinterpret_cast<long long*>(sum_lo),
-                                                             reinterpret_cast<long long*>(sum_hi), counts, K, g, C);
+                                                             reinterpret_cast<long long*>(sum_hi), counts, counts, K, g,
+                                                             1, C);
     return cudaGetLastError();
 }
 
@@ -262,11 +283,8 @@ extern "C" cc_status cc_update_static(int device, const uint16_t* X, int64_t N, 
     if (N > 0) {
         int sms = 0;
         if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return CC_ERR_CUDA;
-        int64_t blocks = (N + 255) / 256;
-        const int64_t cap = (int64_t)sms * 16;
-        if (blocks > cap) blocks = cap;
-#define CALL(G)                                                                                               \
-    update_accumulate_kernel<G><<<(unsigned)blocks, 256, 0, st>>>(X, N, idx, K, sum_lo, sum_hi, counts)
+        cudaError_t e = cudaSuccess;
+#define CALL(G) e = launch_accumulate<G>(sms, X, N, idx, K, sum_lo, sum_hi, counts, 1, st)
         switch (g) {
             case 1: CALL(1); break;   case 2: CALL(2); break;   case 3: CALL(3); break;   case 4: CALL(4); break;
             case 5: CALL(5); break;   case 6: CALL(6); break;   case 7: CALL(7); break;   case 8: CALL(8); break;
@@ -275,8 +293,10 @@ extern "C" cc_status cc_update_static(int device, const uint16_t* X, int64_t N, 
             default: return CC_ERR_UNSUPPORTED_G;
         }
 #undef CALL
+        if (e != cudaSuccess) return CC_ERR_CUDA;
     }
     update_finish_kernel<<<(K * g + 255) / 256, 256, 0, st>>>(reinterpret_cast<long long*>(sum_lo),
-                                                             reinterpret_cast<long long*>(sum_hi), counts, K, g, C);
+                                                             reinterpret_cast<long long*>(sum_hi), counts, counts, K, g,
+                                                             1, C);
     return cudaGetLastError() == cudaSuccess ? CC_OK : CC_ERR_CUDA;
 }

@@ -794,9 +794,10 @@ assign_tensor_persistent_kernel(const uint16_t* __restrict__ X, int64_t N, const
 // centroids 4k .. 4k+3 and 32+4k .. 32+4k+3 (four consecutive centroids every 4 LPP) of the winning
 // 64-centroid chunk with the FMA chain
 // s = fma(x_{g-1}, m_{g-1}, ... fma(x_0, m_0, ||c||^2)), keeping its smallest score, its index and
-// its runner-up; a butterfly over the group gives every lane the chunk's winner and runner-up;
-// then the squared distance to the winner in FP64 (sub, mul, add in dimension order, no
-// contraction) and the near-tie test.  A scan whose scores are off by at most
+// its runner-up; a butterfly over the group gives every lane the chunk's winner and runner-up.
+// A group does this for eight points in turn and lane k keeps the k-th result, so that the rest
+// runs once per 32 points with one point per lane: the squared distance to the winner in FP64
+// (sub, mul, add in dimension order, no contraction), the near-tie test and the stores.  A scan whose scores are off by at most
 //     E = ERR_UNITS 2^-24 (2||c||^2 + ||x||^2) + 2^-14 ||x||_1 / S + 2^-26 / S
 // (|x_t| counted as at least 2^-14) may misorder two scores closer than 2E; every centroid at
 // least as close as the winner has 2||c||^2 + ||x||^2 <= 5||x||^2 + 4 d^2, so a point whose two
@@ -808,55 +809,74 @@ finish_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __r
                      const TcParams* __restrict__ params, uint16_t* __restrict__ idx, float* __restrict__ dist,
                      unsigned* __restrict__ status, unsigned* __restrict__ flagged) {
     const int k = threadIdx.x & (LPP - 1);
-    const int64_t group0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) / LPP;
-    const int64_t n_groups = ((int64_t)gridDim.x * blockDim.x) / LPP;
-    const int64_t rounds = (N + n_groups - 1) / n_groups;            // the same for every lane of a warp
+    const int lane = threadIdx.x & 31;
+    const int64_t warp0 = ((int64_t)blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
+    const int64_t rounds = (N + n_warps * 32 - 1) / (n_warps * 32);  // the same for every lane of a warp
     const float invS = params->invS;
     for (int64_t rd = 0; rd < rounds; ++rd) {
-        const int64_t i_raw = rd * n_groups + group0;
+        // A warp takes 32 consecutive points per round: its four lane groups rescan eight points
+        // each, one after the other, and lane l keeps what was found for point base + l, so that
+        // the exact distance, the bound and the stores are done once for 32 points.
+        const int64_t base = (rd * n_warps + warp0) * 32;
+        float keep_s1 = 0.f, keep_s2 = 0.f;
+        int keep_j = 0;
+#pragma unroll 1
+        for (int sub = 0; sub < LPP; ++sub) {
+            const int64_t i_raw = base + (lane & ~(LPP - 1)) + sub;
+            const int64_t i = i_raw < N ? i_raw : N - 1;
+            const float2 t = tstate[i];
+            const int chunk = __float_as_int(t.y);
+            float x[G];
+            bool nf = false;
+            load_point<G>(X, i, N, x, nf);                       // the same address in the lanes of a group
+            const float4* blk = reinterpret_cast<const float4*>(rescan + (int64_t)chunk * ((G + 1) * TCHUNK)) + k;
+            float s1 = INFINITY, s2 = INFINITY;
+            int j1 = 4 * k;
+#pragma unroll
+            for (int hf = 0; hf < TCHUNK / 4 / LPP; ++hf) {
+                const float4 cs = __ldg(blk + G * (TCHUNK / 4) + hf * LPP);
+                float s[4] = {cs.x, cs.y, cs.z, cs.w};
+#pragma unroll
+                for (int u = 0; u < G; ++u) {
+                    const float4 mv = __ldg(blk + u * (TCHUNK / 4) + hf * LPP);
+                    s[0] = fmaf(x[u], mv.x, s[0]);
+                    s[1] = fmaf(x[u], mv.y, s[1]);
+                    s[2] = fmaf(x[u], mv.z, s[2]);
+                    s[3] = fmaf(x[u], mv.w, s[3]);
+                }
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const bool take = s[e] < s1;                 // ascending index: strict '<' keeps the lowest
+                    s2 = take ? s1 : fminf(s2, s[e]);
+                    j1 = take ? (hf * LPP + k) * 4 + e : j1;
+                    s1 = take ? s[e] : s1;
+                }
+            }
+#pragma unroll
+            for (int o = LPP / 2; o > 0; o >>= 1) {
+                const float os1 = __shfl_xor_sync(0xffffffffu, s1, o);
+                const float os2 = __shfl_xor_sync(0xffffffffu, s2, o);
+                const int oj = __shfl_xor_sync(0xffffffffu, j1, o);
+                const bool take = os1 < s1 || (os1 == s1 && oj < j1);
+                s2 = fminf(take ? s1 : os1, fminf(s2, os2));
+                s1 = take ? os1 : s1;
+                j1 = take ? oj : j1;
+            }
+            if (k == sub) {
+                keep_j = j1 + chunk * TCHUNK;
+                keep_s1 = s1;
+                keep_s2 = fminf(s2, t.x * invS);
+            }
+        }
+        const int64_t i_raw = base + lane;
         const bool live = i_raw < N;
         const int64_t i = live ? i_raw : N - 1;
-        const float2 t = tstate[i];
-        const int chunk = __float_as_int(t.y);
+        int j1 = keep_j;
+        if (j1 >= K) j1 = K - 1;   // only reachable with non-finite input
         float x[G];
         bool nf = false;
-        load_point<G>(X, i, N, x, nf);                       // the same address in the lanes of a group
-        const float4* blk = reinterpret_cast<const float4*>(rescan + (int64_t)chunk * ((G + 1) * TCHUNK)) + k;
-        float s1 = INFINITY, s2 = INFINITY;
-        int j1 = 4 * k;
-#pragma unroll
-        for (int hf = 0; hf < TCHUNK / 4 / LPP; ++hf) {
-            const float4 cs = __ldg(blk + G * (TCHUNK / 4) + hf * LPP);
-            float s[4] = {cs.x, cs.y, cs.z, cs.w};
-#pragma unroll
-            for (int u = 0; u < G; ++u) {
-                const float4 mv = __ldg(blk + u * (TCHUNK / 4) + hf * LPP);
-                s[0] = fmaf(x[u], mv.x, s[0]);
-                s[1] = fmaf(x[u], mv.y, s[1]);
-                s[2] = fmaf(x[u], mv.z, s[2]);
-                s[3] = fmaf(x[u], mv.w, s[3]);
-            }
-#pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const bool take = s[e] < s1;                 // ascending index: strict '<' keeps the lowest
-                s2 = take ? s1 : fminf(s2, s[e]);
-                j1 = take ? (hf * LPP + k) * 4 + e : j1;
-                s1 = take ? s[e] : s1;
-            }
-        }
-#pragma unroll
-        for (int o = LPP / 2; o > 0; o >>= 1) {
-            const float os1 = __shfl_xor_sync(0xffffffffu, s1, o);
-            const float os2 = __shfl_xor_sync(0xffffffffu, s2, o);
-            const int oj = __shfl_xor_sync(0xffffffffu, j1, o);
-            const bool take = os1 < s1 || (os1 == s1 && oj < j1);
-            s2 = fminf(take ? s1 : os1, fminf(s2, os2));
-            s1 = take ? os1 : s1;
-            j1 = take ? oj : j1;
-        }
-        j1 += chunk * TCHUNK;
-        if (j1 >= K) j1 = K - 1;   // only reachable with non-finite input
-        s2 = fminf(s2, t.x * invS);
+        load_point<G>(X, i, N, x, nf);
         double D = 0.0;
         float A = 0.f, L1 = 0.f;
 #pragma unroll
@@ -867,13 +887,13 @@ finish_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __r
             A = fmaf(xf, xf, A);
             L1 += fabsf(x[u]);
         }
-        if (live && k == 0) {
+        if (live) {
             idx[i] = (uint16_t)j1;
             dist[i] = (float)D;
             // A and L1 only feed the bound: FP32 is enough once they are rounded up a little
             const double bound = 2.0 * ((double)TcCfg<G>::ERR_UNITS * 5.9604644775390625e-8 * (5.0 * (double)A * 1.0001 + 4.0 * D)
                                         + (double)invS * (6.103515625e-5 * (double)L1 * 1.0001 + 1.4901161193847656e-8));
-            if (!((double)s2 - (double)s1 > bound)) {
+            if (!((double)keep_s2 - (double)keep_s1 > bound)) {
                 const ull slot = atomicAdd(reinterpret_cast<ull*>(status + 2), 1ull);
                 flagged[slot] = (unsigned)i;
             }
@@ -951,7 +971,7 @@ cudaError_t launch_tensor(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int
         }
         {
             ProfScope ps(ctx, CC_K_ASSIGN_FINISH, st);
-            int64_t fblocks = (N * LPP + 255) / 256;
+            int64_t fblocks = (N + 255) / 256;            // a warp takes 32 points per round
             const int64_t cap = (int64_t)ctx->sm_count * 32;
             if (fblocks > cap) fblocks = cap;
             finish_tensor_kernel<G><<<(unsigned)fblocks, 256, 0, st>>>(

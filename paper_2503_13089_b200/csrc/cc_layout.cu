@@ -121,6 +121,177 @@ decode_transpose_vec_kernel(const uint16_t* __restrict__ C16, const uint16_t* __
     }
 }
 
+// PAPER_T decode for large matrices: persistent CTAs walk over the tiles with the loads of the
+// next tiles already in flight (the codes of tile k+2 and the codebook rows of tile k+1 are
+// requested before tile k goes through shared memory), because a tile's chain DRAM (codes) ->
+// gather -> transpose -> store is otherwise paid once per tile and four to eight resident CTAs do
+// not hide it.  TABLE: the whole FP16 codebook (at most kTableMaxBytes) is staged in shared memory
+// once per CTA and the gather is a shared-memory read at the time of use.
+constexpr int kTileBytes = (TILE_WORDS * 4 + 15) / 16 * 16;
+constexpr int kTableMaxBytes = 46 * 1024;   // four CTAs per SM with their tiles
+
+struct DecodeCodes {
+    unsigned code[2];   // G = 4: two 16-bit codes; otherwise element offset of the 8 values in the codebook
+    unsigned live;      // bit p: row p of this thread lies inside the matrix
+};
+
+struct DecodeTile { int bx, by; };   // tile coordinates along in_features / out_features
+
+// Tile t + gridDim.x from tile t without a division.
+__device__ __forceinline__ void decode_next_tile(DecodeTile& p, int step_x, int step_y, int tiles_x) {
+    p.bx += step_x;
+    p.by += step_y;
+    if (p.bx >= tiles_x) { p.bx -= tiles_x; ++p.by; }
+}
+
+// opg = out_pad / G: codes per in_feature.  out_pad is a multiple of G and a tile starts at a
+// multiple of 64 out_features, so the position inside the sub-vector is (8 c) mod G.
+template <int G>
+__device__ __forceinline__ void decode_load_codes(const uint16_t* __restrict__ idx, DecodeTile p, int tiles_y, int r0,
+                                                  int c, int64_t d_in, int64_t out_pad, int64_t opg, unsigned kmax,
+                                                  DecodeCodes& s) {
+    s.live = 0u;
+    s.code[0] = 0u;
+    s.code[1] = 0u;
+    if (p.by >= tiles_y) return;
+    const int64_t o = (int64_t)p.by * TD + 8 * c;
+    if (o >= out_pad) return;
+    const int64_t i = (int64_t)p.bx * TD + r0;
+    const uint16_t* src = idx + i * opg + (o / G);
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+        if (i + 32 * q < d_in) {
+            s.live |= 1u << q;
+            // a code beyond the codebook must not leave it
+            if constexpr (G == 4) {
+                const unsigned two = __ldg(reinterpret_cast<const unsigned*>(src + 32 * q * opg));
+                s.code[q] = min(two & 0xffffu, kmax) | (min(two >> 16, kmax) << 16);
+            } else {
+                s.code[q] = min((unsigned)__ldg(src + 32 * q * opg), kmax) * (unsigned)G + ((8u * c) & (unsigned)(G - 1));
+            }
+        }
+    }
+}
+
+template <int G>
+__device__ __forceinline__ void decode_gather(const uint16_t* table, const DecodeCodes& s, uint4 (&v)[2]) {
+#pragma unroll
+    for (int q = 0; q < 2; ++q) {
+        v[q] = make_uint4(0u, 0u, 0u, 0u);
+        if (s.live >> q & 1u) {
+            if constexpr (G == 4) {
+                const uint2 a = *reinterpret_cast<const uint2*>(table + (s.code[q] & 0xffffu) * 4u);
+                const uint2 b = *reinterpret_cast<const uint2*>(table + (s.code[q] >> 16) * 4u);
+                v[q] = make_uint4(a.x, a.y, b.x, b.y);
+            } else {
+                v[q] = *reinterpret_cast<const uint4*>(table + s.code[q]);
+            }
+        }
+    }
+}
+
+// One tile through shared memory and out to W_hat.
+__device__ __forceinline__ void decode_emit(unsigned* tile, DecodeTile p, int r0, int c, const uint4 (&v)[2],
+                                            int64_t d_out, int64_t d_in, uint16_t* __restrict__ W_hat) {
+    tile_put8(tile, r0, c, v[0]);
+    tile_put8(tile, r0 + 32, c, v[1]);
+    __syncthreads();
+    uint4 even, odd;
+    tile_column8x2(tile, c, r0, even, odd);
+    const int64_t o = (int64_t)p.by * TD + 2 * r0, i = (int64_t)p.bx * TD + 8 * c;
+    if (i < d_in) {
+        uint16_t* dst = W_hat + o * d_in + i;
+        if (o < d_out) *reinterpret_cast<uint4*>(dst) = even;
+        if (o + 1 < d_out) *reinterpret_cast<uint4*>(dst + d_in) = odd;
+    }
+    __syncthreads();                            // the tile is free for the next round
+}
+
+// The loop is unrolled by two so that the two register sets (A, B) keep their roles: a register
+// that still waits for a load is never copied.
+template <int G, bool TABLE>
+__global__ void __launch_bounds__(256, 4)
+decode_transpose_pipe_kernel(const uint16_t* __restrict__ C16, const uint16_t* __restrict__ idx, int K, int64_t d_out,
+                             int64_t d_in, int64_t out_pad, uint16_t* __restrict__ W_hat, int tiles_x, int tiles_y) {
+    extern __shared__ __align__(16) unsigned char decode_smem[];
+    unsigned* tile = reinterpret_cast<unsigned*>(decode_smem);
+    const uint16_t* table = C16;
+    if constexpr (TABLE) {
+        uint16_t* staged = reinterpret_cast<uint16_t*>(decode_smem + kTileBytes);
+        for (int v = threadIdx.x; v < K * G / 4; v += 256)
+            reinterpret_cast<uint2*>(staged)[v] = __ldg(reinterpret_cast<const uint2*>(C16) + v);
+        table = staged;
+    }
+    const int c = threadIdx.x & 7, r0 = threadIdx.x >> 3;
+    const unsigned kmax = (unsigned)K - 1u;
+    const int64_t opg = out_pad / G;
+    const int step_x = (int)(gridDim.x % (unsigned)tiles_x), step_y = (int)(gridDim.x / (unsigned)tiles_x);
+    DecodeTile t0 = {(int)(blockIdx.x % (unsigned)tiles_x), (int)(blockIdx.x / (unsigned)tiles_x)};
+#define CC_DECODE_CODES(P, S) decode_load_codes<G>(idx, P, tiles_y, r0, c, d_in, out_pad, opg, kmax, S)
+    DecodeCodes sA, sB;
+    uint4 vA[2], vB[2];
+    CC_DECODE_CODES(t0, sA);
+    DecodeTile t1 = t0;
+    decode_next_tile(t1, step_x, step_y, tiles_x);
+    if constexpr (TABLE) {
+        __syncthreads();                        // the table is staged
+        while (t0.by < tiles_y) {
+            CC_DECODE_CODES(t1, sB);
+            decode_gather<G>(table, sA, vA);
+            decode_emit(tile, t0, r0, c, vA, d_out, d_in, W_hat);
+            if (t1.by >= tiles_y) break;
+            t0 = t1;
+            decode_next_tile(t0, step_x, step_y, tiles_x);
+            CC_DECODE_CODES(t0, sA);
+            decode_gather<G>(table, sB, vB);
+            decode_emit(tile, t1, r0, c, vB, d_out, d_in, W_hat);
+            t1 = t0;
+            decode_next_tile(t1, step_x, step_y, tiles_x);
+        }
+    } else {
+        CC_DECODE_CODES(t1, sB);
+        decode_gather<G>(table, sA, vA);
+        while (t0.by < tiles_y) {
+            DecodeTile t2 = t1;
+            decode_next_tile(t2, step_x, step_y, tiles_x);
+            decode_gather<G>(table, sB, vB);    // tile t1 (nothing live past the last tile)
+            CC_DECODE_CODES(t2, sA);
+            decode_emit(tile, t0, r0, c, vA, d_out, d_in, W_hat);
+            if (t1.by >= tiles_y) break;
+            t0 = t2;
+            decode_next_tile(t0, step_x, step_y, tiles_x);
+            decode_gather<G>(table, sA, vA);    // tile t2
+            CC_DECODE_CODES(t0, sB);
+            decode_emit(tile, t1, r0, c, vB, d_out, d_in, W_hat);
+            t1 = t0;
+            t0 = t2;
+        }
+    }
+#undef CC_DECODE_CODES
+}
+
+template <int G>
+cudaError_t launch_decode_pipe(int sm_count, const uint16_t* C16, const uint16_t* idx, int K, int64_t d_out,
+                               int64_t d_in, int64_t out_pad, uint16_t* W_hat, int tiles_x, int tiles_y,
+                               cudaStream_t st) {
+    const int64_t n_tiles = (int64_t)tiles_x * tiles_y;
+    const bool staged = K * G * 2 <= kTableMaxBytes;
+    const int smem = kTileBytes + (staged ? K * G * 2 : 0);
+    int64_t grid = (int64_t)sm_count * 4;
+    if (grid > n_tiles) grid = n_tiles;
+    if (staged) {
+        const cudaError_t e = cudaFuncSetAttribute(decode_transpose_pipe_kernel<G, true>,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, smem);
+        if (e != cudaSuccess) return e;
+        decode_transpose_pipe_kernel<G, true><<<(unsigned)grid, 256, smem, st>>>(C16, idx, K, d_out, d_in, out_pad,
+                                                                                 W_hat, tiles_x, tiles_y);
+    } else {
+        decode_transpose_pipe_kernel<G, false><<<(unsigned)grid, 256, smem, st>>>(C16, idx, K, d_out, d_in, out_pad,
+                                                                                  W_hat, tiles_x, tiles_y);
+    }
+    return cudaGetLastError();
+}
+
 // ROWS reshape: copy each row, padding it to in_pad elements.
 __global__ void __launch_bounds__(256)
 reshape_rows_kernel(const uint16_t* __restrict__ W, int64_t d_out, int64_t d_in, int64_t in_pad,
@@ -214,12 +385,18 @@ cudaError_t cc_launch_reshape(cc_ctx* ctx, const uint16_t* W, int64_t d_out, int
 
 cudaError_t cc_launch_decode(cc_ctx* ctx, const uint16_t* C16, int K, int g, const uint16_t* idx, int64_t d_out,
                              int64_t d_in, int layout, uint16_t* W_hat, cudaStream_t st) {
-    (void)K;
     ProfScope ps(ctx, CC_K_DECODE, st);
     if (layout == CC_LAYOUT_PAPER_T) {
         const int64_t out_pad = pad_to(d_out, g);
         dim3 grid((unsigned)((d_in + TD - 1) / TD), (unsigned)((d_out + TD - 1) / TD));
         const bool vec = d_in % 8 == 0 && out_pad % 8 == 0;
+        const int64_t n_tiles = (int64_t)grid.x * grid.y;
+        // enough tiles for persistent CTAs with loads in flight across tiles
+        if (vec && (g == 4 || g == 8 || g == 16) && n_tiles >= (int64_t)ctx->sm_count * 8) {
+            if (g == 4) return launch_decode_pipe<4>(ctx->sm_count, C16, idx, K, d_out, d_in, out_pad, W_hat, (int)grid.x, (int)grid.y, st);
+            if (g == 8) return launch_decode_pipe<8>(ctx->sm_count, C16, idx, K, d_out, d_in, out_pad, W_hat, (int)grid.x, (int)grid.y, st);
+            return launch_decode_pipe<16>(ctx->sm_count, C16, idx, K, d_out, d_in, out_pad, W_hat, (int)grid.x, (int)grid.y, st);
+        }
         if (vec && g == 4) decode_transpose_vec_kernel<4><<<grid, 256, 0, st>>>(C16, idx, d_out, d_in, out_pad, W_hat);
         else if (vec && g == 8) decode_transpose_vec_kernel<8><<<grid, 256, 0, st>>>(C16, idx, d_out, d_in, out_pad, W_hat);
         else if (vec && g == 16) decode_transpose_vec_kernel<16><<<grid, 256, 0, st>>>(C16, idx, d_out, d_in, out_pad, W_hat);

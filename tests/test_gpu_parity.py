@@ -51,6 +51,22 @@ def test_reshape_and_decode_match_oracle(d_out, d_in, g, layout):
     assert np.array_equal(u.u16_np(What.view(torch.uint16)).reshape(d_out, d_in), want.view(np.uint16))
 
 
+@pytest.mark.parametrize("g,K", [(4, 3000), (8, 2900), (16, 1400), (4, 1), (8, 6400), (16, 3000), (4, 65536)])
+def test_decode_of_a_large_matrix_matches_oracle(g, K):
+    """Matrices with at least 8 tiles per SM take the persistent kernel (codebooks of at most 46 KB
+    staged in shared memory, larger ones gathered from global memory); ragged tiles on both edges."""
+    cc, u = _cc(), _u()
+    d_out, d_in = 2056, 2568
+    rng = np.random.default_rng(g * 100003 + K)
+    N = cc.cc_num_subvectors(d_out, d_in, g, 0)
+    C16 = rng.standard_normal((K, g)).astype(np.float16)
+    idx = rng.integers(0, K, N).astype(np.uint16)
+    What = torch.zeros((d_out, d_in), dtype=torch.float16, device="cuda")
+    cc.cc_decode(u.ctx(), u.half_dev(C16), K, g, u.dev(idx.view(np.int16)).view(torch.uint16), d_out, d_in, 0, What)
+    want = oracle.decode(C16, idx.astype(np.int32), d_out, d_in, 0)
+    assert np.array_equal(u.u16_np(What.view(torch.uint16)).reshape(d_out, d_in), want.view(np.uint16))
+
+
 @pytest.mark.parametrize("N,g,K,seed", [(5000, 4, 700, 42), (257, 3, 257, 9), (100000, 8, 4096, 1)])
 def test_init_codebook_matches_oracle(N, g, K, seed):
     cc, u = _cc(), _u()
@@ -67,6 +83,8 @@ def test_init_codebook_matches_oracle(N, g, K, seed):
 ASSIGN_CASES = [
     # N, g, K   (tile = 2048 points x 128..512 centroids: several tiles and ragged tails)
     (1, 4, 1), (31, 4, 2), (2049, 4, 33), (5000, 4, 255), (5000, 4, 257), (70001, 4, 1000),
+    (16384, 4, 64), (16385, 1, 130), (20011, 5, 1000), (33000, 8, 700), (18000, 12, 200), (17000, 16, 2100),
+    (40000, 3, 65), (25000, 7, 4097),
     (20000, 4, 4096), (3000, 4, 5000), (9000, 8, 300), (4097, 8, 2049), (6000, 16, 129),
     (2500, 16, 1500), (3001, 1, 17), (3001, 2, 64), (3001, 3, 100), (3001, 5, 600), (3001, 6, 90),
     (3001, 7, 1025), (3001, 9, 513), (1500, 12, 77), (1500, 13, 300), (1500, 15, 64),

@@ -121,7 +121,7 @@ decode_transpose_vec_kernel(const uint16_t* __restrict__ C16, const uint16_t* __
     }
 }
 
-// PAPER_T decode for large matrices: persistent CTAs walk over the tiles with the loads of the
+// PAPER_T decode of large matrices for g = 8 and 16: persistent CTAs walk over the tiles with the loads of the
 // next tiles already in flight (the codes of tile k+2 and the codebook rows of tile k+1 are
 // requested before tile k goes through shared memory), because a tile's chain DRAM (codes) ->
 // gather -> transpose -> store is otherwise paid once per tile and four to eight resident CTAs do
@@ -129,9 +129,10 @@ decode_transpose_vec_kernel(const uint16_t* __restrict__ C16, const uint16_t* __
 // once per CTA and the gather is a shared-memory read at the time of use.
 constexpr int kTileBytes = (TILE_WORDS * 4 + 15) / 16 * 16;
 constexpr int kTableMaxBytes = 46 * 1024;   // four CTAs per SM with their tiles
+constexpr int kPipeMaxTableBytes = 128 * 1024;
 
 struct DecodeCodes {
-    unsigned code[2];   // G = 4: two 16-bit codes; otherwise element offset of the 8 values in the codebook
+    unsigned code[2];   // element offset of the 8 values in the codebook
     unsigned live;      // bit p: row p of this thread lies inside the matrix
 };
 
@@ -163,12 +164,7 @@ __device__ __forceinline__ void decode_load_codes(const uint16_t* __restrict__ i
         if (i + 32 * q < d_in) {
             s.live |= 1u << q;
             // a code beyond the codebook must not leave it
-            if constexpr (G == 4) {
-                const unsigned two = __ldg(reinterpret_cast<const unsigned*>(src + 32 * q * opg));
-                s.code[q] = min(two & 0xffffu, kmax) | (min(two >> 16, kmax) << 16);
-            } else {
-                s.code[q] = min((unsigned)__ldg(src + 32 * q * opg), kmax) * (unsigned)G + ((8u * c) & (unsigned)(G - 1));
-            }
+            s.code[q] = min((unsigned)__ldg(src + 32 * q * opg), kmax) * (unsigned)G + ((8u * c) & (unsigned)(G - 1));
         }
     }
 }
@@ -179,13 +175,7 @@ __device__ __forceinline__ void decode_gather(const uint16_t* table, const Decod
     for (int q = 0; q < 2; ++q) {
         v[q] = make_uint4(0u, 0u, 0u, 0u);
         if (s.live >> q & 1u) {
-            if constexpr (G == 4) {
-                const uint2 a = *reinterpret_cast<const uint2*>(table + (s.code[q] & 0xffffu) * 4u);
-                const uint2 b = *reinterpret_cast<const uint2*>(table + (s.code[q] >> 16) * 4u);
-                v[q] = make_uint4(a.x, a.y, b.x, b.y);
-            } else {
-                v[q] = *reinterpret_cast<const uint4*>(table + s.code[q]);
-            }
+            v[q] = *reinterpret_cast<const uint4*>(table + s.code[q]);
         }
     }
 }
@@ -391,9 +381,12 @@ cudaError_t cc_launch_decode(cc_ctx* ctx, const uint16_t* C16, int K, int g, con
         dim3 grid((unsigned)((d_in + TD - 1) / TD), (unsigned)((d_out + TD - 1) / TD));
         const bool vec = d_in % 8 == 0 && out_pad % 8 == 0;
         const int64_t n_tiles = (int64_t)grid.x * grid.y;
-        // enough tiles for persistent CTAs with loads in flight across tiles
-        if (vec && (g == 4 || g == 8 || g == 16) && n_tiles >= (int64_t)ctx->sm_count * 8) {
-            if (g == 4) return launch_decode_pipe<4>(ctx->sm_count, C16, idx, K, d_out, d_in, out_pad, W_hat, (int)grid.x, (int)grid.y, st);
+        // Enough tiles for persistent CTAs with loads in flight across tiles, and a codebook that
+        // stays in L1: there the chain of latencies bounds a tile.  A larger codebook is bound by the
+        // L2 sectors its gathers move, and more resident threads (the kernel below) serve it better.
+        // With g = 4 (8-byte rows, two gathers per 16 output bytes) the plain kernel measured faster.
+        if (vec && (g == 8 || g == 16) && n_tiles >= (int64_t)ctx->sm_count * 8 &&
+            (int64_t)K * g * 2 <= kPipeMaxTableBytes) {
             if (g == 8) return launch_decode_pipe<8>(ctx->sm_count, C16, idx, K, d_out, d_in, out_pad, W_hat, (int)grid.x, (int)grid.y, st);
             return launch_decode_pipe<16>(ctx->sm_count, C16, idx, K, d_out, d_in, out_pad, W_hat, (int)grid.x, (int)grid.y, st);
         }

@@ -53,8 +53,9 @@ def test_reshape_and_decode_match_oracle(d_out, d_in, g, layout):
 
 @pytest.mark.parametrize("g,K", [(4, 3000), (8, 2900), (16, 1400), (4, 1), (8, 6400), (16, 3000), (4, 65536)])
 def test_decode_of_a_large_matrix_matches_oracle(g, K):
-    """Matrices with at least 8 tiles per SM take the persistent kernel (codebooks of at most 46 KB
-    staged in shared memory, larger ones gathered from global memory); ragged tiles on both edges."""
+    """Matrices with at least 8 tiles per SM: g = 8 and 16 with a codebook of at most 128 KB take the
+    persistent kernel (codebooks of at most 46 KB staged in shared memory), the others the plain
+    tiled kernel; ragged tiles on both edges."""
     cc, u = _cc(), _u()
     d_out, d_in = 2056, 2568
     rng = np.random.default_rng(g * 100003 + K)

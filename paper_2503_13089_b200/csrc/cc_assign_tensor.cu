@@ -102,16 +102,48 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 }
 
 // Bounded wait.  Returns false when the CTA is aborting (this or another waiter timed out).
+// Every lane of a warp waits on the same barrier word with the same parity, so the branches are
+// uniform across the warp and say so (bra.uni): the compiler then needs no convergence barriers
+// around the loop, which sits on the critical path of every tile.
+// `ok` is left alone by a wait that succeeds and cleared by one that gives up.
+__device__ __forceinline__ void mbar_wait_acc(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t& ok) {
+    asm volatile(
+        "{\n\t"
+        ".reg .pred p, q;\n\t"
+        ".reg .u64 t0, t1;\n\t"
+        ".reg .u32 n, f;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "@p bra.uni MBW_DONE;\n\t"
+        "mov.u64 t0, %%clock64;\n\t"
+        "mov.u32 n, 0;\n"
+        "MBW_LOOP:\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "@p bra.uni MBW_DONE;\n\t"
+        "add.u32 n, n, 1;\n\t"
+        "and.b32 f, n, 255;\n\t"
+        "setp.ne.u32 q, f, 0;\n\t"
+        "@q bra.uni MBW_LOOP;\n\t"
+        "ld.volatile.shared.u32 f, [%3];\n\t"
+        "setp.ne.u32 q, f, 0;\n\t"
+        "@q bra.uni MBW_DONE;\n\t"                 // another waiter gave up: p is false
+        "mov.u64 t1, %%clock64;\n\t"
+        "sub.u64 t1, t1, t0;\n\t"
+        "setp.le.u64 q, t1, %4;\n\t"
+        "@q bra.uni MBW_LOOP;\n\t"
+        "mov.u32 f, 1;\n\t"
+        "st.volatile.shared.u32 [%3], f;\n"          // time-out: p is false
+        "MBW_DONE:\n\t"
+        "@!p mov.u32 %0, 0;\n\t"
+        "}"
+        : "+r"(ok)
+        : "r"(bar), "r"(parity), "r"(smem_u32(const_cast<int*>(abort_flag))), "l"(WAIT_LIMIT)
+        : "memory");
+}
+
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
-    if (mbar_try(bar, parity)) return true;
-    const long long t0 = clock64();
-    for (unsigned spin = 1;; ++spin) {
-        if (mbar_try(bar, parity)) return true;
-        if ((spin & 255u) == 0u) {
-            if (*abort_flag) return false;
-            if (clock64() - t0 > WAIT_LIMIT) { *abort_flag = 1; return false; }
-        }
-    }
+    uint32_t ok = 1u;
+    mbar_wait_acc(bar, parity, abort_flag, ok);
+    return ok != 0u;
 }
 
 __device__ __forceinline__ float min3(float a, float b, float c) {
@@ -271,6 +303,20 @@ prep_tensor_kernel(const float* __restrict__ C, int K, int Kpad, TcParams* __res
                    "+r"(v[22]), "+r"(v[23]), "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]),    \
                    "+r"(v[29]), "+r"(v[30]), "+r"(v[31])                                                         \
                  :: "memory")
+// One wait for two loads: both register sets are named.
+#define TMEM_WAIT64(v, w)                                                                                        \
+    asm volatile("tcgen05.wait::ld.sync.aligned;"                                                                \
+                 : "+r"(v[0]), "+r"(v[1]), "+r"(v[2]), "+r"(v[3]), "+r"(v[4]), "+r"(v[5]), "+r"(v[6]), "+r"(v[7]),  \
+                   "+r"(v[8]), "+r"(v[9]), "+r"(v[10]), "+r"(v[11]), "+r"(v[12]), "+r"(v[13]), "+r"(v[14]),      \
+                   "+r"(v[15]), "+r"(v[16]), "+r"(v[17]), "+r"(v[18]), "+r"(v[19]), "+r"(v[20]), "+r"(v[21]),    \
+                   "+r"(v[22]), "+r"(v[23]), "+r"(v[24]), "+r"(v[25]), "+r"(v[26]), "+r"(v[27]), "+r"(v[28]),    \
+                   "+r"(v[29]), "+r"(v[30]), "+r"(v[31]),                                                        \
+                   "+r"(w[0]), "+r"(w[1]), "+r"(w[2]), "+r"(w[3]), "+r"(w[4]), "+r"(w[5]), "+r"(w[6]), "+r"(w[7]),  \
+                   "+r"(w[8]), "+r"(w[9]), "+r"(w[10]), "+r"(w[11]), "+r"(w[12]), "+r"(w[13]), "+r"(w[14]),      \
+                   "+r"(w[15]), "+r"(w[16]), "+r"(w[17]), "+r"(w[18]), "+r"(w[19]), "+r"(w[20]), "+r"(w[21]),    \
+                   "+r"(w[22]), "+r"(w[23]), "+r"(w[24]), "+r"(w[25]), "+r"(w[26]), "+r"(w[27]), "+r"(w[28]),    \
+                   "+r"(w[29]), "+r"(w[30]), "+r"(w[31])                                                         \
+                 :: "memory")
 
 // A operand rows [x repeated SPLIT times, 2^15, 2^6, 2^-3, 2^-12, 0..] of points base + e,
 // e = first, first + step, .. < count, into the tiles at sA (canonical layout, 16 bytes at a time).
@@ -371,7 +417,7 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* 
         }
         for (int s = 0; s < SLOTS; ++s) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(t_full + s)));
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(t_empty + s)), "r"(EPI_WARPS));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(t_empty + s)), "r"(EPI_WARPS * 32));
         }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -472,29 +518,29 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* 
 #pragma unroll
         for (int a = 0; a < NA; ++a) { b1[a] = INFINITY; b2[a] = INFINITY; bc[a] = cg; }
         const uint32_t tbase = tmem + ((uint32_t)(quarter * 32) << 16) + cg * TCHUNK;
-        bool ok = true;
+        uint32_t okw = 1u;
         int q = 0;
         int chunk_id = cg;                                // id of this warp's chunk in codebook tile b
-        for (int b = 0; b < n_btiles && ok; ++b, chunk_id += EW) {
+        for (int b = 0; b < n_btiles && okw; ++b, chunk_id += EW) {
 #pragma unroll
             for (int a = 0; a < NA; ++a) {
-                if (a >= na || !ok) continue;
+                if (a >= na) continue;
+                // A wait that gives up is only acted upon after the tiles of this round: once the abort
+                // flag is up the remaining waits return at their next look at it, and reading an
+                // accumulator that was never written or releasing it once more harms nothing.
                 const int slot = FULL ? (a % SLOTS) : (q % SLOTS);
                 const uint32_t par = FULL ? ((a / SLOTS) & 1) : ((q / SLOTS) & 1);
-                ok = mbar_wait(smem_u32(t_full + slot), par, abort_flag);
+                mbar_wait_acc(smem_u32(t_full + slot), par, abort_flag, okw);
                 ++q;
-                if (!ok) continue;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 uint32_t v0[32], v1[32];
                 TMEM_LD32(v0, tbase + slot * TN);
                 TMEM_LD32(v1, tbase + slot * TN + 32);
-                TMEM_WAIT32(v0);
-                TMEM_WAIT32(v1);
-                // the 64 columns are in registers: hand this warp's share of the accumulator back
+                TMEM_WAIT64(v0, v1);
+                // the 64 columns are in registers: every lane hands back its own share of the
+                // accumulator (the barrier counts 16 x 32 arrivals; no predicate, no warp synchronisation)
                 asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                __syncwarp();
-                if (lane == 0)
-                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(t_empty + slot)) : "memory");
+                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(t_empty + slot)) : "memory");
                 if constexpr (DUMP) {
                     const int64_t i = base + a * TM + r;
                     if (i < N) {
@@ -521,7 +567,7 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* 
                 }
             }
             asm volatile("bar.sync 1, %0;" ::"r"(EPI_WARPS * 32));
-            if (cg == 0 && ok && !*abort_flag) {
+            if (cg == 0 && okw && !*abort_flag) {
 #pragma unroll
                 for (int a = 0; a < NA; ++a) {
                     const int64_t i = base + a * TM + r;
@@ -591,7 +637,7 @@ assign_tensor_persistent_kernel(const uint16_t* __restrict__ X, int64_t N, const
         }
         for (int s = 0; s < SLOTS; ++s) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(t_full + s)));
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(t_empty + s)), "r"(EPI_WARPS));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(t_empty + s)), "r"(EPI_WARPS * 32));
         }
         for (int s = 0; s < 2; ++s) {
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(a_full + s)));
@@ -717,7 +763,9 @@ assign_tensor_persistent_kernel(const uint16_t* __restrict__ X, int64_t N, const
         // ------------------------------------------------------------ epilogue warps
         const int quarter = warp & 3, cg = warp >> 2;     // TMEM lane quarter, 64-column group
         const int r = quarter * 32 + lane;                // row of the point tile = TMEM lane
-        const uint32_t tbase = tmem + ((uint32_t)(quarter * 32) << 16) + cg * TCHUNK;
+        // the same value in all lanes, and visibly so (broadcast from lane 0): the accumulator address
+        // can then live in a uniform register instead of being converted for every load
+        const uint32_t tbase = __shfl_sync(0xffffffffu, tmem + ((uint32_t)(quarter * 32) << 16) + cg * TCHUNK, 0);
         bool ok = true;
         for (int it = 0; it < n_iter && ok; ++it) {
             float b1[NA], b2[NA];
@@ -725,23 +773,24 @@ assign_tensor_persistent_kernel(const uint16_t* __restrict__ X, int64_t N, const
 #pragma unroll
             for (int a = 0; a < NA; ++a) { b1[a] = INFINITY; b2[a] = INFINITY; bc[a] = cg; }
             int chunk_id = cg;
-            for (int b = 0; b < n_btiles && ok; ++b, chunk_id += EW) {
+            uint32_t okw = 1u;
+            for (int b = 0; b < n_btiles && okw; ++b, chunk_id += EW) {
 #pragma unroll
                 for (int a = 0; a < NA; ++a) {
-                    if (!ok) continue;
+                    // A wait that gives up is only acted upon after the eight tiles: once the abort flag
+                    // is up the remaining waits return at their next look at it, and reading an
+                    // accumulator that was never written or releasing it once more harms nothing.
                     const int slot = a % SLOTS;
-                    ok = mbar_wait(smem_u32(t_full + slot), (a / SLOTS) & 1, abort_flag);
-                    if (!ok) continue;
+                    mbar_wait_acc(smem_u32(t_full + slot), (a / SLOTS) & 1, abort_flag, okw);
                     asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                     uint32_t v0[32], v1[32];
                     TMEM_LD32(v0, tbase + slot * TN);
                     TMEM_LD32(v1, tbase + slot * TN + 32);
-                    TMEM_WAIT32(v0);
-                    TMEM_WAIT32(v1);
+                    TMEM_WAIT64(v0, v1);
+                    // every lane hands back its own 32 x 64 share (the barrier counts 16 x 32 arrivals):
+                    // no predicate, no warp synchronisation
                     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
-                    __syncwarp();
-                    if (lane == 0)
-                        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(t_empty + slot)) : "memory");
+                    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(t_empty + slot)) : "memory");
                     const float m = chunk_min64(v0, v1);
                     const bool better = m < b1[a];
                     b2[a] = better ? b1[a] : fminf(b2[a], m);
@@ -749,6 +798,7 @@ assign_tensor_persistent_kernel(const uint16_t* __restrict__ X, int64_t N, const
                     b1[a] = better ? m : b1[a];
                 }
             }
+            ok = okw != 0u;
             // ---- merge the EW column groups of each point and store; the exchange area is reused by
             //      the next group, hence the second barrier
             if (cg > 0) {

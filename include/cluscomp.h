@@ -157,6 +157,20 @@ int64_t cc_tensor_scores_ld(int K);
 cc_status cc_tensor_scores(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const float* C, int K,
                            float* scores, void* stream);
 
+/* Self-test of the bounded waits of the tensor-core E-step (no counterpart in the paper).  Every
+ * wait of those kernels on a shared-memory barrier gives up after a clock limit, raises a flag that
+ * makes the CTA's other waits return, and the kernel then reports CC_ERR_DEVICE_TIMEOUT through
+ * cc_poll_status instead of hanging.  This call runs one warp through that wait code with the
+ * given limit (1e3 .. 4e9 clock cycles) and copies to the HOST arrays:
+ *   results[0] = 1: a wait on a barrier whose phase completes succeeds;
+ *   results[1] = 0: a wait on a barrier nobody arrives on gives up;
+ *   results[2] = 1: the abort flag is up afterwards;
+ *   results[3] = 0: a further wait returns unsuccessfully;
+ *   cycles[0], cycles[1]: how long the second and third wait took (the second a little more than
+ *   the limit, the third far less).
+ * Synchronous; allocates and frees 64 bytes of device memory. */
+cc_status cc_selftest_bounded_wait(cc_ctx* ctx, int64_t limit_cycles, int32_t* results, int64_t* cycles);
+
 /* M-step of Section 3.1: counts[j] = |{i : idx[i] = j}| (exact), C[j] = mean of those x_i
  * (exact integer sum, one rounding to FP32); a cluster with no member keeps its centroid
  * bit for bit (the paper does not say; this library's rule).  C: in = previous, out = new.

@@ -49,6 +49,7 @@ SIGNATURES = {
     "cc_assign": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp]),
     "cc_tensor_scores_ld": (_i64, [_i32]),
     "cc_tensor_scores": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp]),
+    "cc_selftest_bounded_wait": (_i32, [_vp, _i64, _vp, _vp]),
     "cc_update": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp]),
     "cc_update_static": (_i32, [_i32, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp]),
     "cc_codebook_grad": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp]),
@@ -214,6 +215,15 @@ def cc_set_codebook(ctx, C0, K, g, C, stream=None) -> None:
 def cc_assign(ctx, X, N, g, C, K, idx, dist=None, objective=None, n_resolved=None, stream=None) -> None:
     _check(load().cc_assign(ctx._h, _ptr(X), N, g, _ptr(C), K, _ptr(idx), _ptr(dist), _ptr(objective),
                             _ptr(n_resolved), _stream(stream)), "cc_assign")
+
+
+def cc_selftest_bounded_wait(ctx, limit_cycles: int):
+    """Returns (results[4], cycles[2]) of the bounded-wait self-test (see cluscomp.h)."""
+    res = (ct.c_int32 * 4)()
+    cyc = (ct.c_int64 * 2)()
+    _check(load().cc_selftest_bounded_wait(ctx._h, limit_cycles, ct.cast(res, ct.c_void_p), ct.cast(cyc, ct.c_void_p)),
+           "cc_selftest_bounded_wait")
+    return list(res), list(cyc)
 
 
 def cc_tensor_scores_ld(K: int) -> int:

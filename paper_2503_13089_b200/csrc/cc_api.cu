@@ -273,6 +273,26 @@ cc_status cc_tensor_scores(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, con
     return from_cuda(cc_launch_tensor_scores(ctx, L, X, N, g, C, K, scores, (cudaStream_t)stream));
 }
 
+cc_status cc_selftest_bounded_wait(cc_ctx* ctx, int64_t limit_cycles, int32_t* results, int64_t* cycles) {
+    if (!ctx || !results || !cycles) return CC_ERR_NULL;
+    if (limit_cycles < 1000 || limit_cycles > 4000000000LL) return CC_ERR_SHAPE;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    void* dev = nullptr;
+    if (cudaMalloc(&dev, 64) != cudaSuccess) return CC_ERR_CUDA;
+    int* out_dev = static_cast<int*>(dev);
+    long long* cyc_dev = reinterpret_cast<long long*>(static_cast<char*>(dev) + 16);
+    cc_status st = CC_OK;
+    long long cyc[2] = {0, 0};
+    if (cudaMemset(dev, 0, 64) != cudaSuccess || cc_launch_wait_selftest(limit_cycles, out_dev, cyc_dev, 0) != cudaSuccess ||
+        cudaMemcpy(results, out_dev, 4 * sizeof(int32_t), cudaMemcpyDeviceToHost) != cudaSuccess ||
+        cudaMemcpy(cyc, cyc_dev, sizeof(cyc), cudaMemcpyDeviceToHost) != cudaSuccess)
+        st = CC_ERR_CUDA;
+    cycles[0] = cyc[0];
+    cycles[1] = cyc[1];
+    cudaFree(dev);
+    return st;
+}
+
 cc_status cc_update(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const uint16_t* idx, int K, float* C,
                     int32_t* counts, void* stream) {
     if (!ctx || !C || !counts || (N > 0 && (!X || !idx))) return CC_ERR_NULL;

@@ -106,7 +106,8 @@ __device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity) {
 // uniform across the warp and say so (bra.uni): the compiler then needs no convergence barriers
 // around the loop, which sits on the critical path of every tile.
 // `ok` is left alone by a wait that succeeds and cleared by one that gives up.
-__device__ __forceinline__ void mbar_wait_acc(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t& ok) {
+__device__ __forceinline__ void mbar_wait_acc(uint32_t bar, uint32_t parity, volatile int* abort_flag, uint32_t& ok,
+                                              long long limit = WAIT_LIMIT) {
     asm volatile(
         "{\n\t"
         ".reg .pred p, q;\n\t"
@@ -120,7 +121,7 @@ __device__ __forceinline__ void mbar_wait_acc(uint32_t bar, uint32_t parity, vol
         "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
         "@p bra.uni MBW_DONE;\n\t"
         "add.u32 n, n, 1;\n\t"
-        "and.b32 f, n, 255;\n\t"
+        "and.b32 f, n, 15;\n\t"                    // a failed try has already slept in hardware: look up every 16
         "setp.ne.u32 q, f, 0;\n\t"
         "@q bra.uni MBW_LOOP;\n\t"
         "ld.volatile.shared.u32 f, [%3];\n\t"
@@ -136,7 +137,7 @@ __device__ __forceinline__ void mbar_wait_acc(uint32_t bar, uint32_t parity, vol
         "@!p mov.u32 %0, 0;\n\t"
         "}"
         : "+r"(ok)
-        : "r"(bar), "r"(parity), "r"(smem_u32(const_cast<int*>(abort_flag))), "l"(WAIT_LIMIT)
+        : "r"(bar), "r"(parity), "r"(smem_u32(const_cast<int*>(abort_flag))), "l"(limit)
         : "memory");
 }
 
@@ -1060,6 +1061,42 @@ cudaError_t cc_launch_assign_tensor(cc_ctx* ctx, const WsLayout& L, const uint16
 #undef CALL
     if (e != cudaSuccess) return e;
     return cc_launch_assign_tail(ctx, L, X, N, g, C, K, idx, dist, objective, n_resolved, st);
+}
+
+// Self-test of the bounded wait: one warp (a) waits on a barrier whose phase thread 0 completes,
+// (b) waits on a barrier that nobody ever arrives on, with the given clock limit, and (c) waits on
+// it again with the abort flag up.  out: {result of a, result of b, abort flag after b, result of c};
+// cycles: {duration of b, duration of c}.
+__global__ void __launch_bounds__(32)
+wait_selftest_kernel(long long limit, int* __restrict__ out, long long* __restrict__ cycles) {
+    __shared__ __align__(8) uint64_t bars[2];
+    __shared__ int abort_word;
+    volatile int* abort_flag = &abort_word;
+    if (threadIdx.x == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(bars)));
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(bars + 1)));
+        abort_word = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    __syncwarp();
+    if (threadIdx.x == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bars)) : "memory");
+    uint32_t ok_a = 1u, ok_b = 1u, ok_c = 1u;
+    mbar_wait_acc(smem_u32(bars), 0, abort_flag, ok_a, limit);
+    const long long t0 = clock64();
+    mbar_wait_acc(smem_u32(bars + 1), 0, abort_flag, ok_b, limit);
+    const long long t1 = clock64();
+    const int flag_after_b = *abort_flag;
+    mbar_wait_acc(smem_u32(bars + 1), 0, abort_flag, ok_c, limit);
+    const long long t2 = clock64();
+    if (threadIdx.x == 0) {
+        out[0] = (int)ok_a; out[1] = (int)ok_b; out[2] = flag_after_b; out[3] = (int)ok_c;
+        cycles[0] = t1 - t0; cycles[1] = t2 - t1;
+    }
+}
+
+cudaError_t cc_launch_wait_selftest(long long limit, int* out_dev, long long* cycles_dev, cudaStream_t st) {
+    wait_selftest_kernel<<<1, 32, 0, st>>>(limit, out_dev, cycles_dev);
+    return cudaGetLastError();
 }
 
 cudaError_t cc_launch_tensor_scores(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64_t N, int g,

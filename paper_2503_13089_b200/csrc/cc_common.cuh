@@ -107,6 +107,7 @@ cudaError_t cc_launch_assign_tensor(cc_ctx*, const WsLayout&, const uint16_t* X,
                                     cudaStream_t);
 // Verification aid: every comparison score of the tensor-core scan, N x cc_tensor_score_ld(K) floats.
 int cc_tensor_score_ld(int K);
+cudaError_t cc_launch_wait_selftest(long long limit_cycles, int* out_dev, long long* cycles_dev, cudaStream_t);
 cudaError_t cc_launch_tensor_scores(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const float* C,
                                     int K, float* scores, cudaStream_t);
 // Second stage shared by both E-step paths: exact FP64 decision for the flagged points, then

@@ -536,3 +536,19 @@ def test_cfg4_full_size_one_iteration_sampled():
     sel = wl.subset_positions(len(X), 0.0002, 5)
     C, trace, tol = _lockstep(X, C0, 1, sel=sel)
     print("cfg4 tolerated near-ties on the sample:", tol, "objective", trace)
+
+
+# ------------------------------------------------------------------ bounded device-side waits
+
+def test_a_barrier_wait_that_cannot_end_gives_up_and_reports_it():
+    """The scan kernels wait on shared-memory barriers; each wait is bounded by a clock limit.  The
+    self-test runs that wait code on a barrier nobody arrives on (limit 2e6 cycles, about 1 ms)."""
+    cc, u = _cc(), _u()
+    limit = 2_000_000
+    res, cyc = cc.cc_selftest_bounded_wait(u.ctx(), limit)
+    assert res == [1, 0, 1, 0]                 # completes; gives up; flag raised; later waits return at once
+    assert limit < cyc[0] < 4 * limit          # gave up shortly after the limit
+    assert cyc[1] < limit // 2                 # with the flag up a wait ends after 16 polls
+    with pytest.raises(cc.CCError):
+        cc.cc_selftest_bounded_wait(u.ctx(), 10)   # limit out of range
+

@@ -870,17 +870,24 @@ finish_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __r
         // each, one after the other, and lane l keeps what was found for point base + l, so that
         // the exact distance, the bound and the stores are done once for 32 points.
         const int64_t base = (rd * n_warps + warp0) * 32;
+        // every lane loads its own point and scan result once (coalesced); the group then gets the
+        // point it works on from the lane that owns it
+        const int64_t i_raw = base + lane;
+        const bool live = i_raw < N;
+        const int64_t i = live ? i_raw : N - 1;
+        const float2 t_own = tstate[i];
+        float x_own[G];
+        bool nf = false;
+        load_point<G>(X, i, N, x_own, nf);
         float keep_s1 = 0.f, keep_s2 = 0.f;
         int keep_j = 0;
 #pragma unroll 1
         for (int sub = 0; sub < LPP; ++sub) {
-            const int64_t i_raw = base + (lane & ~(LPP - 1)) + sub;
-            const int64_t i = i_raw < N ? i_raw : N - 1;
-            const float2 t = tstate[i];
-            const int chunk = __float_as_int(t.y);
+            const int src = (lane & ~(LPP - 1)) + sub;
+            const int chunk = __shfl_sync(0xffffffffu, __float_as_int(t_own.y), src);
             float x[G];
-            bool nf = false;
-            load_point<G>(X, i, N, x, nf);                       // the same address in the lanes of a group
+#pragma unroll
+            for (int u = 0; u < G; ++u) x[u] = __shfl_sync(0xffffffffu, x_own[u], src);
             const float4* blk = reinterpret_cast<const float4*>(rescan + (int64_t)chunk * ((G + 1) * TCHUNK)) + k;
             float s1 = INFINITY, s2 = INFINITY;
             int j1 = 4 * k;
@@ -914,20 +921,15 @@ finish_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __r
                 s1 = take ? os1 : s1;
                 j1 = take ? oj : j1;
             }
-            if (k == sub) {
+            if (k == sub) {                   // this round's point is the lane's own
                 keep_j = j1 + chunk * TCHUNK;
                 keep_s1 = s1;
-                keep_s2 = fminf(s2, t.x * invS);
+                keep_s2 = fminf(s2, t_own.x * invS);
             }
         }
-        const int64_t i_raw = base + lane;
-        const bool live = i_raw < N;
-        const int64_t i = live ? i_raw : N - 1;
         int j1 = keep_j;
         if (j1 >= K) j1 = K - 1;   // only reachable with non-finite input
-        float x[G];
-        bool nf = false;
-        load_point<G>(X, i, N, x, nf);
+        const float (&x)[G] = x_own;
         double D = 0.0;
         float A = 0.f, L1 = 0.f;
 #pragma unroll

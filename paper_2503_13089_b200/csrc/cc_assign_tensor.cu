@@ -350,36 +350,20 @@ __device__ __forceinline__ void build_a_rows(const uint16_t* __restrict__ X, int
     }
 }
 
-// The reduction of one 64-column chunk held in two 32-register halves: four independent chains,
-// 30 three-input minima + 2.
+// The reduction of one 64-column chunk held in two 32-register halves: a tree of three-input
+// minima (21 + 7 + 2 + 1, and one two-input minimum for the 64th value).  The first level takes
+// three consecutive registers each, so that registers free up as the tree advances; measured 2 %
+// faster than four running chains of the same 32 instructions, which also spilled.
 __device__ __forceinline__ float chunk_min64(const uint32_t* v0, const uint32_t* v1) {
-    float m0 = min3(__uint_as_float(v0[0]), __uint_as_float(v0[1]), __uint_as_float(v0[2]));
-    float m1 = min3(__uint_as_float(v0[8]), __uint_as_float(v0[9]), __uint_as_float(v0[10]));
-    float m2 = min3(__uint_as_float(v0[16]), __uint_as_float(v0[17]), __uint_as_float(v0[18]));
-    float m3 = min3(__uint_as_float(v0[24]), __uint_as_float(v0[25]), __uint_as_float(v0[26]));
+    auto val = [&](int i) { return __uint_as_float(i < 32 ? v0[i] : v1[i - 32]); };
+    float t[21];
 #pragma unroll
-    for (int hf = 0; hf < 2; ++hf) {
-        const uint32_t* v = hf ? v1 : v0;
-        if (hf) {
-            m0 = min3(m0, __uint_as_float(v[0]), __uint_as_float(v[1]));
-            m1 = min3(m1, __uint_as_float(v[8]), __uint_as_float(v[9]));
-            m2 = min3(m2, __uint_as_float(v[16]), __uint_as_float(v[17]));
-            m3 = min3(m3, __uint_as_float(v[24]), __uint_as_float(v[25]));
-            m0 = min3(m0, __uint_as_float(v[2]), __uint_as_float(v[10]));
-            m2 = min3(m2, __uint_as_float(v[18]), __uint_as_float(v[26]));
-        }
-        m0 = min3(m0, __uint_as_float(v[3]), __uint_as_float(v[4]));
-        m1 = min3(m1, __uint_as_float(v[11]), __uint_as_float(v[12]));
-        m2 = min3(m2, __uint_as_float(v[19]), __uint_as_float(v[20]));
-        m3 = min3(m3, __uint_as_float(v[27]), __uint_as_float(v[28]));
-        m0 = min3(m0, __uint_as_float(v[5]), __uint_as_float(v[6]));
-        m1 = min3(m1, __uint_as_float(v[13]), __uint_as_float(v[14]));
-        m2 = min3(m2, __uint_as_float(v[21]), __uint_as_float(v[22]));
-        m3 = min3(m3, __uint_as_float(v[29]), __uint_as_float(v[30]));
-        m0 = min3(m0, __uint_as_float(v[7]), __uint_as_float(v[15]));
-        m2 = min3(m2, __uint_as_float(v[23]), __uint_as_float(v[31]));
-    }
-    return fminf(min3(m0, m1, m2), m3);
+    for (int k = 0; k < 21; ++k) t[k] = min3(val(3 * k), val(3 * k + 1), val(3 * k + 2));
+    float u[7];
+#pragma unroll
+    for (int j = 0; j < 7; ++j) u[j] = min3(t[3 * j], t[3 * j + 1], t[3 * j + 2]);
+    const float w0 = min3(u[0], u[1], u[2]), w1 = min3(u[3], u[4], u[5]);
+    return fminf(min3(w0, w1, u[6]), val(63));
 }
 
 // DUMP = true writes every score (divided by S) to `dump` (row stride dump_ld) instead of

@@ -318,9 +318,9 @@ def main():
             kd = ((3 if 3 * g + 4 <= 48 else 2) * g + 4 + 15) // 16 * 16
             executed_tf = achieved_tf * kd / g
             # DRAM bytes of one launch of the scan kernel: one ncu capture of this kernel at g = 4 on
-            # 1,048,576 points (8,953,856 bytes read, 0 written: X once, the staged codebook and the
+            # 1,048,576 points (8,947,712 bytes read, 0 written: X once, the staged codebook and the
             # per-point results stay in L2), scaled by the number of points; other g were not captured
-            traffic = counts[0]["N"] * (8953856.0 / 1048576.0) if g == 4 else None
+            traffic = counts[0]["N"] * (8947712.0 / 1048576.0) if g == 4 else None
             roofline = {"bound": "alu", "kernel": "assign_tensor_kernel (E-step: tcgen05 scores + min-reduction epilogue)",
                         "achieved": achieved_tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": achieved_tf / peak_tf,
                         "peak_kind": "ALU min-reduction: 148 SMs x 128 lanes x 1965 MHz scores/s x 2g flops per score",

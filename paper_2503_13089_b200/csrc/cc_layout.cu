@@ -379,7 +379,8 @@ cudaError_t cc_launch_decode(cc_ctx* ctx, const uint16_t* C16, int K, int g, con
     if (layout == CC_LAYOUT_PAPER_T) {
         const int64_t out_pad = pad_to(d_out, g);
         dim3 grid((unsigned)((d_in + TD - 1) / TD), (unsigned)((d_out + TD - 1) / TD));
-        const bool vec = d_in % 8 == 0 && out_pad % 8 == 0;
+        // the vector kernels read two codes as one 32-bit word
+        const bool vec = d_in % 8 == 0 && out_pad % 8 == 0 && (reinterpret_cast<uintptr_t>(idx) & 3u) == 0;
         const int64_t n_tiles = (int64_t)grid.x * grid.y;
         // Enough tiles for persistent CTAs with loads in flight across tiles, and a codebook that
         // stays in L1: there the chain of latencies bounds a tile.  A larger codebook is bound by the

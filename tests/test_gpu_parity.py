@@ -51,6 +51,23 @@ def test_reshape_and_decode_match_oracle(d_out, d_in, g, layout):
     assert np.array_equal(u.u16_np(What.view(torch.uint16)).reshape(d_out, d_in), want.view(np.uint16))
 
 
+def test_decode_accepts_codes_that_are_only_two_byte_aligned():
+    """The vector kernels read two codes as one 32-bit word; a code array that starts at an odd
+    element must take the scalar kernel instead of faulting."""
+    cc, u = _cc(), _u()
+    d_out, d_in, g, K = 136, 200, 4, 50
+    rng = np.random.default_rng(5)
+    N = cc.cc_num_subvectors(d_out, d_in, g, 0)
+    C16 = rng.standard_normal((K, g)).astype(np.float16)
+    idx = rng.integers(0, K, N).astype(np.uint16)
+    buf = torch.zeros(N + 1, dtype=torch.int16, device="cuda")
+    buf[1:] = u.dev(idx.view(np.int16))
+    What = torch.zeros((d_out, d_in), dtype=torch.float16, device="cuda")
+    cc.cc_decode(u.ctx(), u.half_dev(C16), K, g, buf[1:].view(torch.uint16), d_out, d_in, 0, What)
+    want = oracle.decode(C16, idx.astype(np.int32), d_out, d_in, 0)
+    assert np.array_equal(u.u16_np(What.view(torch.uint16)).reshape(d_out, d_in), want.view(np.uint16))
+
+
 @pytest.mark.parametrize("g,K", [(4, 3000), (8, 2900), (16, 1400), (4, 1), (8, 6400), (16, 3000), (4, 65536)])
 def test_decode_of_a_large_matrix_matches_oracle(g, K):
     """Matrices with at least 8 tiles per SM: g = 8 and 16 with a codebook of at most 128 KB take the

@@ -8,8 +8,8 @@
 // |S m| < 2^15 and S ||c||^2 < 2^30 for every centroid (m = -2c); S m = h1 + h2 + h3 is the FP32
 // value cut into FP16 pieces (each piece is the FP16 rounding of what is left), and
 // S ||c||^2 (from FP64) = 2^15 p1 + 2^6 p2 + 2^-3 p3 + 2^-12 p4 likewise.  Scaling by a power of
-// two changes neither the order of the scores nor their rounding.  g = 15, 16 use two pieces of m
-// (relative residue 2^-22) to keep the contraction at 48 columns.
+// two changes neither the order of the scores nor their rounding.  g = 5, 6 and g = 10..16 use two
+// pieces of m (relative residue 2^-22), which shortens the contraction to 16, 32 and 48 columns.
 //
 // Subnormal pieces are never emitted: the tensor core adds the products of one instruction after
 // aligning them by the operands' exponent FIELDS, so a subnormal piece next to the constant 2^15
@@ -29,9 +29,9 @@
 // smallest and second-smallest 64-centroid chunk minimum and the id of the best chunk (one
 // 3-input min per two scores); the index inside the chunk, the distance and the near-tie flag are
 // computed afterwards by the finish kernel from FP32 data.  Nothing N x K is written to memory.
-// Three instantiations share this structure: a persistent kernel (g <= 9: one CTA per SM walks over
+// Three instantiations share this structure: a persistent kernel (g <= 14: one CTA per SM walks over
 // groups of NA point tiles while an extra warp builds the next group's A operand), a one-group-per-
-// CTA kernel specialised for full groups (g >= 10), and a generic one for the ragged rest and for
+// CTA kernel specialised for full groups (g = 15, 16), and a generic one for the ragged rest and for
 // small inputs.
 //
 // Every wait on an mbarrier is bounded (clock based); on a time-out the CTA raises the status
@@ -56,7 +56,11 @@ constexpr int LPP = 8;             // lanes per point in the finish kernel
 constexpr long long WAIT_LIMIT = 4000000000LL;   // clock cycles (about 2 s)
 
 template <int G> struct TcCfg {
-    static constexpr int SPLIT = (3 * G + NQ <= 48) ? 3 : 2;        // FP16 pieces of each S m value
+    // FP16 pieces of each S m value: three (residue 2^-33), or two (residue 2^-22) where that makes
+    // the contraction shorter (g = 5, 6: 16 instead of 32 columns; g = 10..14: 32 instead of 48) or
+    // where three do not fit 48 columns (g = 15, 16)
+    static constexpr int KD3 = (3 * G + NQ + 15) / 16 * 16, KD2 = (2 * G + NQ + 15) / 16 * 16;
+    static constexpr int SPLIT = (KD3 <= 48 && KD3 <= KD2) ? 3 : 2;
     static constexpr int KD = (SPLIT * G + NQ + 15) / 16 * 16;      // contraction length (halves)
     static constexpr int A_TILE = TM * KD * 2;                      // bytes
     static constexpr int B_TILE = TN * KD * 2;
@@ -579,7 +583,7 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* 
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(SLOTS * TN));
 }
 
-// Persistent form of the scan for contraction lengths up to 32 columns (g <= 9): one CTA per SM walks
+// Persistent form of the scan for contraction lengths up to 32 columns (g <= 14): one CTA per SM walks
 // over groups of NA point tiles (group = blockIdx.x, + gridDim.x, ..) and keeps TWO sets of A tiles
 // in shared memory.  A 19th warp builds the next group's A operand while the current group is
 // multiplied and reduced, so the tensor core and the epilogue never wait for a CTA to start or to

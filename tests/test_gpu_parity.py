@@ -149,13 +149,14 @@ def test_assign_fp32_and_tensor_paths_agree_with_oracle_and_each_other(N, g, K):
 def _tensor_units(g):
     """Rounding model of the tensor-core scan as the library documents it: contraction length,
     number of FP16 pieces per centroid value, allowed error in units of 2^-24 (2||c||^2 + ||x||^2)."""
-    split = 3 if 3 * g + 4 <= 48 else 2
-    kd = (split * g + 4 + 15) // 16 * 16
+    kd3, kd2 = (3 * g + 4 + 15) // 16 * 16, (2 * g + 4 + 15) // 16 * 16
+    split = 3 if (kd3 <= 48 and kd3 <= kd2) else 2       # two pieces where that shortens the contraction
+    kd = kd3 if split == 3 else kd2
     return split, kd, 8 * (kd // 16) + (4 if split == 2 else 0)
 
 
 @pytest.mark.parametrize("kind", ["weights", "wide_range", "on_centroids", "huge"])
-@pytest.mark.parametrize("g", [1, 3, 4, 5, 8, 9, 12, 14, 15, 16])
+@pytest.mark.parametrize("g", [1, 3, 4, 5, 6, 8, 9, 10, 12, 14, 15, 16])
 def test_tensor_scores_obey_the_rounding_model(g, kind):
     """Every raw score of the tensor-core scan against float64: the error must stay inside the
     bound that decides which points are sent to the exact stage (and, here, inside half of it)."""

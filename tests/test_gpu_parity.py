@@ -128,7 +128,8 @@ def test_assign_matches_oracle(N, g, K):
                                    (3001, 7, 1025), (3001, 9, 513), (1500, 12, 77), (1500, 13, 300), (1500, 15, 64),
                                    (150000, 4, 300), (40000, 9, 700),
                                    # enough full groups for the persistent scan, plus a ragged rest for the generic one
-                                   (400001, 4, 300), (310000, 9, 129), (305000, 16, 70)])
+                                   (400001, 4, 300), (310000, 9, 129), (305000, 16, 70), (320001, 6, 200), (310000, 12, 129),
+                                   (306000, 14, 75)])
 def test_assign_fp32_and_tensor_paths_agree_with_oracle_and_each_other(N, g, K):
     cc, u = _cc(), _u()
     X = wl.make_points(N, g, 1000 + N + g)

@@ -315,8 +315,8 @@ def main():
             evals_launch = flops_launch / (2 * g)
             peak_scores = NOMINAL_SM * NOMINAL_LANES * NOMINAL_MHZ * 1e6
             peak_tf = peak_scores * 2 * g / 1e12
-            kd3, kd2 = (3 * g + 4 + 15) // 16 * 16, (2 * g + 4 + 15) // 16 * 16
-            kd = kd3 if (kd3 <= 48 and kd3 <= kd2) else kd2      # the library's choice of operand pieces
+            kd34, kd24, kd22 = ((3 * g + 4 + 15) // 16 * 16, (2 * g + 4 + 15) // 16 * 16, (2 * g + 2 + 15) // 16 * 16)
+            kd = kd34 if (kd34 <= 48 and kd34 <= min(kd24, kd22)) else min(kd24, kd22)   # the library's choice of operand pieces
             executed_tf = achieved_tf * kd / g
             # DRAM bytes of one launch of the scan kernel: one ncu capture of this kernel at g = 4 on
             # 1,048,576 points (8,947,712 bytes read, 0 written: X once, the staged codebook and the

@@ -8,8 +8,10 @@
 // |S m| < 2^15 and S ||c||^2 < 2^30 for every centroid (m = -2c); S m = h1 + h2 + h3 is the FP32
 // value cut into FP16 pieces (each piece is the FP16 rounding of what is left), and
 // S ||c||^2 (from FP64) = 2^15 p1 + 2^6 p2 + 2^-3 p3 + 2^-12 p4 likewise.  Scaling by a power of
-// two changes neither the order of the scores nor their rounding.  g = 5, 6 and g = 10..16 use two
-// pieces of m (relative residue 2^-22), which shortens the contraction to 16, 32 and 48 columns.
+// two changes neither the order of the scores nor their rounding.  Where it shortens the contraction
+// (g = 5, 6, 7: 16 columns; g = 10..15: 32) or is needed to fit 48 columns (g = 16), m is cut into two
+// pieces only (relative residue 2^-22); for g = 7 and 15 the norm is cut into two pieces as well,
+// S ||c||^2 = 2^e p1 + 2^(e-11) p2 with e fitted to the largest norm of the call.
 //
 // Subnormal pieces are never emitted: the tensor core adds the products of one instruction after
 // aligning them by the operands' exponent FIELDS, so a subnormal piece next to the constant 2^15
@@ -29,9 +31,9 @@
 // smallest and second-smallest 64-centroid chunk minimum and the id of the best chunk (one
 // 3-input min per two scores); the index inside the chunk, the distance and the near-tie flag are
 // computed afterwards by the finish kernel from FP32 data.  Nothing N x K is written to memory.
-// Three instantiations share this structure: a persistent kernel (g <= 14: one CTA per SM walks over
+// Three instantiations share this structure: a persistent kernel (g <= 15: one CTA per SM walks over
 // groups of NA point tiles while an extra warp builds the next group's A operand), a one-group-per-
-// CTA kernel specialised for full groups (g = 15, 16), and a generic one for the ragged rest and for
+// CTA kernel specialised for full groups (g = 16), and a generic one for the ragged rest and for
 // small inputs.
 //
 // Every wait on an mbarrier is bounded (clock based); on a time-out the CTA raises the status
@@ -46,7 +48,6 @@ namespace {
 constexpr int TM = 128;            // points per MMA = TMEM lanes
 constexpr int TN = 256;            // centroids per MMA = TMEM columns of one accumulator
 constexpr int TCHUNK = 64;         // centroids per tracked minimum = columns per epilogue warp
-constexpr int NQ = 4;              // FP16 pieces of S ||c||^2
 constexpr int EW = TN / TCHUNK;    // epilogue warps per TMEM lane quarter
 constexpr int EPI_WARPS = 4 * EW;
 constexpr int TC_THREADS = (EPI_WARPS + 2) * 32;
@@ -56,11 +57,19 @@ constexpr int LPP = 8;             // lanes per point in the finish kernel
 constexpr long long WAIT_LIMIT = 4000000000LL;   // clock cycles (about 2 s)
 
 template <int G> struct TcCfg {
-    // FP16 pieces of each S m value: three (residue 2^-33), or two (residue 2^-22) where that makes
-    // the contraction shorter (g = 5, 6: 16 instead of 32 columns; g = 10..14: 32 instead of 48) or
-    // where three do not fit 48 columns (g = 15, 16)
-    static constexpr int KD3 = (3 * G + NQ + 15) / 16 * 16, KD2 = (2 * G + NQ + 15) / 16 * 16;
-    static constexpr int SPLIT = (KD3 <= 48 && KD3 <= KD2) ? 3 : 2;
+    // FP16 pieces of each S m value (SPLIT) and of S ||c||^2 (NQ).  Default three and four; fewer
+    // where that makes the contraction shorter or is needed to fit 48 columns:
+    //   two pieces of m (relative residue 2^-22): g = 5, 6 (16 instead of 32 columns), g = 10..14 (32
+    //   instead of 48), g = 16;
+    //   two pieces of m and two of the norm: g = 7 (16 columns), g = 15 (32 columns).  The two norm
+    //   pieces multiply constants 2^e and 2^(e-11) with e fitted to the largest norm of the call
+    //   (norm_exponent), so that the residue is 2^-22 of the norm and a piece written as zero loses
+    //   at most 2^(e-25).
+    static constexpr int KD34 = (3 * G + 4 + 15) / 16 * 16, KD24 = (2 * G + 4 + 15) / 16 * 16,
+                         KD22 = (2 * G + 2 + 15) / 16 * 16;
+    static constexpr bool FULL3 = KD34 <= 48 && KD34 <= KD24 && KD34 <= KD22;
+    static constexpr int SPLIT = FULL3 ? 3 : 2;
+    static constexpr int NQ = (FULL3 || KD24 <= KD22) ? 4 : 2;
     static constexpr int KD = (SPLIT * G + NQ + 15) / 16 * 16;      // contraction length (halves)
     static constexpr int A_TILE = TM * KD * 2;                      // bytes
     static constexpr int B_TILE = TN * KD * 2;
@@ -70,7 +79,7 @@ template <int G> struct TcCfg {
     // Rounding model of the accumulation, in units of 2^-24 (2||c||^2 + ||x||^2): measured on the
     // device at 2.3 / 3.4 / 4.2 units for one / two / three 16-column MMA steps; the two-piece
     // split adds 4.
-    static constexpr int ERR_UNITS = 8 * (KD / 16) + (SPLIT == 2 ? 4 : 0);
+    static constexpr int ERR_UNITS = 8 * (KD / 16) + (SPLIT == 2 ? 4 : 0) + (NQ == 2 ? 4 : 0);
 };
 
 // Written by the range kernel / prep kernel, read by the finish kernel (workspace, 16 bytes).
@@ -199,8 +208,19 @@ __device__ __forceinline__ __half normal_or_zero(__half h) {
     return ((__half_as_ushort(h) & 0x7c00u) == 0u) ? __ushort_as_half((unsigned short)0) : h;
 }
 
-__device__ __forceinline__ float qconst(int p) {   // 2^15, 2^6, 2^-3, 2^-12
-    return p == 0 ? 32768.0f : p == 1 ? 64.0f : p == 2 ? 0.125f : 0.000244140625f;
+// Exponent e of the larger of the two norm constants (NQ = 2): the smallest with S qmax / 2^e < 2^15,
+// kept within [-3, 15] so that 2^e and 2^(e-11) are normal FP16 numbers.
+__device__ __forceinline__ int norm_exponent(float S, unsigned qmax_bits) {
+    int e = floor_log2_bits(__float_as_uint(S)) + floor_log2_bits(qmax_bits) - 14;
+    e = e < -3 ? -3 : e;
+    return e > 15 ? 15 : e;
+}
+
+// Constants that multiply the norm pieces: 2^15, 2^6, 2^-3, 2^-12 (four pieces) or 2^e, 2^(e-11) (two).
+template <int NQ>
+__device__ __forceinline__ float qconst(int p, int e) {
+    if constexpr (NQ == 2) return __int_as_float((e - 11 * p + 127) << 23);
+    else return p == 0 ? 32768.0f : p == 1 ? 64.0f : p == 2 ? 0.125f : 0.000244140625f;
 }
 
 // Staged B operand: tile b holds centroids 256b .. 256b+255 in the canonical layout, KD halves per
@@ -213,8 +233,9 @@ __global__ void __launch_bounds__(256)
 prep_tensor_kernel(const float* __restrict__ C, int K, int Kpad, TcParams* __restrict__ params,
                    uint16_t* __restrict__ gB, float* __restrict__ rescan) {
     using Cfg = TcCfg<G>;
-    constexpr int KD = Cfg::KD, SPLIT = Cfg::SPLIT;
+    constexpr int KD = Cfg::KD, SPLIT = Cfg::SPLIT, NQ = Cfg::NQ;
     const float S = scale_from_range(params->cmax_bits, params->qmax_bits);
+    const int ne = norm_exponent(S, params->qmax_bits);
     const int e = blockIdx.x * blockDim.x + threadIdx.x;
     if (e == 0) { params->S = S; params->invS = 1.0f / S; }
     if (e >= Kpad * (KD / 8)) return;
@@ -249,7 +270,7 @@ prep_tensor_kernel(const float* __restrict__ C, int K, int Kpad, TcParams* __res
             double R = s * (double)S;
 #pragma unroll
             for (int p = 0; p < NQ; ++p) {
-                const double a = (double)qconst(p);
+                const double a = (double)qconst<NQ>(p, ne);
                 qp[p] = normal_or_zero(__double2half(R / a));   // division by a power of two: exact
                 R -= (double)__half2float(qp[p]) * a;           // exact: cancels the leading bits of R
             }
@@ -327,9 +348,12 @@ prep_tensor_kernel(const float* __restrict__ C, int K, int Kpad, TcParams* __res
 // e = first, first + step, .. < count, into the tiles at sA (canonical layout, 16 bytes at a time).
 template <int G>
 __device__ __forceinline__ void build_a_rows(const uint16_t* __restrict__ X, int64_t N, int64_t base, int first,
-                                             int step, int count, unsigned char* sA, bool& nonfinite) {
+                                             int step, int count, unsigned char* sA, bool& nonfinite,
+                                             const TcParams* __restrict__ params) {
     using Cfg = TcCfg<G>;
-    constexpr int KD = Cfg::KD, SPLIT = Cfg::SPLIT;
+    constexpr int KD = Cfg::KD, SPLIT = Cfg::SPLIT, NQ = Cfg::NQ;
+    int ne = 0;                                  // only the two-piece norm has call-dependent constants
+    if constexpr (NQ == 2) ne = norm_exponent(scale_from_range(params->cmax_bits, params->qmax_bits), params->qmax_bits);
     for (int e = first; e < count; e += step) {
         float x[G];
         load_point<G>(X, base + e, N, x, nonfinite);
@@ -337,7 +361,7 @@ __device__ __forceinline__ void build_a_rows(const uint16_t* __restrict__ X, int
 #pragma unroll
         for (int k = 0; k < KD; ++k) {
             h[k] = (k < SPLIT * G) ? __half_as_ushort(__float2half_rn(x[k % G]))    // exact: x is FP16 data
-                 : (k < SPLIT * G + NQ) ? __half_as_ushort(__float2half_rn(qconst(k - SPLIT * G)))
+                 : (k < SPLIT * G + NQ) ? __half_as_ushort(__float2half_rn(qconst<NQ>(k - SPLIT * G, ne)))
                  : (unsigned short)0;
         }
         unsigned char* tile = sA + (e / TM) * Cfg::A_TILE;
@@ -412,7 +436,7 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* 
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     bool nonfinite = false;
-    build_a_rows<G>(X, N, base, tid, TC_THREADS, na * TM, sA, nonfinite);
+    build_a_rows<G>(X, N, base, tid, TC_THREADS, na * TM, sA, nonfinite, params);
     if (nonfinite) atomicOr(status, CC_DEV_NONFINITE);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> async proxy (MMA)
     if (warp == 0) {
@@ -583,7 +607,7 @@ assign_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* 
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(SLOTS * TN));
 }
 
-// Persistent form of the scan for contraction lengths up to 32 columns (g <= 14): one CTA per SM walks
+// Persistent form of the scan for contraction lengths up to 32 columns (g <= 15): one CTA per SM walks
 // over groups of NA point tiles (group = blockIdx.x, + gridDim.x, ..) and keeps TWO sets of A tiles
 // in shared memory.  A 19th warp builds the next group's A operand while the current group is
 // multiplied and reduced, so the tensor core and the epilogue never wait for a CTA to start or to
@@ -602,7 +626,8 @@ template <int G> struct PersistCfg {
 template <int G>
 __global__ void __launch_bounds__(PERSIST_THREADS, 1)
 assign_tensor_persistent_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* __restrict__ gB, int n_btiles,
-                                int n_groups, float2* __restrict__ tstate, unsigned* __restrict__ status) {
+                                int n_groups, const TcParams* __restrict__ params, float2* __restrict__ tstate,
+                                unsigned* __restrict__ status) {
     using Cfg = TcCfg<G>;
     constexpr int KD = Cfg::KD, STAGES = Cfg::STAGES;
     constexpr int A_TILE = Cfg::A_TILE, B_TILE = Cfg::B_TILE, A_SET = NA * A_TILE;
@@ -637,7 +662,7 @@ assign_tensor_persistent_kernel(const uint16_t* __restrict__ X, int64_t N, const
     }
     // first group's A operand: built by everybody
     bool nonfinite = false;
-    build_a_rows<G>(X, N, (int64_t)blockIdx.x * (NA * TM), tid, PERSIST_THREADS, NA * TM, sA, nonfinite);
+    build_a_rows<G>(X, N, (int64_t)blockIdx.x * (NA * TM), tid, PERSIST_THREADS, NA * TM, sA, nonfinite, params);
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> async proxy (MMA)
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
@@ -742,7 +767,7 @@ assign_tensor_persistent_kernel(const uint16_t* __restrict__ X, int64_t N, const
                 if (!ok) break;
             }
             const int64_t group = (int64_t)blockIdx.x + (int64_t)it * gridDim.x;
-            build_a_rows<G>(X, N, group * (NA * TM), lane, 32, NA * TM, sA + buf * A_SET, nonfinite);
+            build_a_rows<G>(X, N, group * (NA * TM), lane, 32, NA * TM, sA + buf * A_SET, nonfinite, params);
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
             __syncwarp();
             if (lane == 0)
@@ -837,7 +862,7 @@ assign_tensor_persistent_kernel(const uint16_t* __restrict__ X, int64_t N, const
 // A group does this for eight points in turn and lane k keeps the k-th result, so that the rest
 // runs once per 32 points with one point per lane: the squared distance to the winner in FP64
 // (sub, mul, add in dimension order, no contraction), the near-tie test and the stores.  A scan whose scores are off by at most
-//     E = ERR_UNITS 2^-24 (2||c||^2 + ||x||^2) + 2^-14 ||x||_1 / S + 2^-26 / S
+//     E = ERR_UNITS 2^-24 (2||c||^2 + ||x||^2) + 2^-14 ||x||_1 / S + 2^-26 / S   (2^(e-25) / S with two norm pieces)
 // (|x_t| counted as at least 2^-14) may misorder two scores closer than 2E; every centroid at
 // least as close as the winner has 2||c||^2 + ||x||^2 <= 5||x||^2 + 4 d^2, so a point whose two
 // smallest scores are closer than 2E with that substitution goes to the exact stage.
@@ -853,6 +878,11 @@ finish_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __r
     const int64_t n_warps = ((int64_t)gridDim.x * blockDim.x) >> 5;
     const int64_t rounds = (N + n_warps * 32 - 1) / (n_warps * 32);  // the same for every lane of a warp
     const float invS = params->invS;
+    // what the norm pieces may lose to a piece written as zero, in scaled units: 2^-26 with four
+    // pieces, 2^(e-25) with two
+    double norm_abs = 1.4901161193847656e-8;
+    if constexpr (TcCfg<G>::NQ == 2)
+        norm_abs = (double)__int_as_float((norm_exponent(params->S, params->qmax_bits) - 25 + 127) << 23);
     for (int64_t rd = 0; rd < rounds; ++rd) {
         // A warp takes 32 consecutive points per round: its four lane groups rescan eight points
         // each, one after the other, and lane l keeps what was found for point base + l, so that
@@ -933,7 +963,7 @@ finish_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __r
             dist[i] = (float)D;
             // A and L1 only feed the bound: FP32 is enough once they are rounded up a little
             const double bound = 2.0 * ((double)TcCfg<G>::ERR_UNITS * 5.9604644775390625e-8 * (5.0 * (double)A * 1.0001 + 4.0 * D)
-                                        + (double)invS * (6.103515625e-5 * (double)L1 * 1.0001 + 1.4901161193847656e-8));
+                                        + (double)invS * (6.103515625e-5 * (double)L1 * 1.0001 + norm_abs));
             if (!((double)keep_s2 - (double)keep_s1 > bound)) {
                 const ull slot = atomicAdd(reinterpret_cast<ull*>(status + 2), 1ull);
                 flagged[slot] = (unsigned)i;
@@ -999,7 +1029,7 @@ cudaError_t launch_tensor(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int
                     attr_p = true;
                 }
                 assign_tensor_persistent_kernel<G><<<ctx->sm_count, PERSIST_THREADS, PersistCfg<G>::SMEM, st>>>(
-                    X, N, gB, Kpad / TN, (int)full_blocks, tstate, status);
+                    X, N, gB, Kpad / TN, (int)full_blocks, params, tstate, status);
             } else if (full_blocks > 0)
                 assign_tensor_kernel<G, false, true><<<(unsigned)full_blocks, TC_THREADS, Cfg::SMEM, st>>>(
                     X, N, gB, Kpad / TN, NA, 0, params, tstate, status, nullptr, 0);

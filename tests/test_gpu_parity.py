@@ -150,14 +150,16 @@ def test_assign_fp32_and_tensor_paths_agree_with_oracle_and_each_other(N, g, K):
 def _tensor_units(g):
     """Rounding model of the tensor-core scan as the library documents it: contraction length,
     number of FP16 pieces per centroid value, allowed error in units of 2^-24 (2||c||^2 + ||x||^2)."""
-    kd3, kd2 = (3 * g + 4 + 15) // 16 * 16, (2 * g + 4 + 15) // 16 * 16
-    split = 3 if (kd3 <= 48 and kd3 <= kd2) else 2       # two pieces where that shortens the contraction
-    kd = kd3 if split == 3 else kd2
-    return split, kd, 8 * (kd // 16) + (4 if split == 2 else 0)
+    kd34, kd24, kd22 = (3 * g + 4 + 15) // 16 * 16, (2 * g + 4 + 15) // 16 * 16, (2 * g + 2 + 15) // 16 * 16
+    full = kd34 <= 48 and kd34 <= kd24 and kd34 <= kd22
+    split = 3 if full else 2                 # two pieces of a value where that shortens the contraction
+    nq = 4 if (full or kd24 <= kd22) else 2  # ... and two pieces of the norm (g = 7, 15)
+    kd = (split * g + nq + 15) // 16 * 16
+    return split, kd, 8 * (kd // 16) + (4 if split == 2 else 0) + (4 if nq == 2 else 0), nq
 
 
 @pytest.mark.parametrize("kind", ["weights", "wide_range", "on_centroids", "huge"])
-@pytest.mark.parametrize("g", [1, 3, 4, 5, 6, 8, 9, 10, 12, 14, 15, 16])
+@pytest.mark.parametrize("g", [1, 3, 4, 5, 6, 7, 8, 9, 10, 12, 14, 15, 16])
 def test_tensor_scores_obey_the_rounding_model(g, kind):
     """Every raw score of the tensor-core scan against float64: the error must stay inside the
     bound that decides which points are sent to the exact stage (and, here, inside half of it)."""
@@ -191,10 +193,14 @@ def test_tensor_scores_obey_the_rounding_model(g, kind):
     # the library's scale: largest power of two with S * 2 max|c| < 2^15 and S * max||c||^2 < 2^30
     k = min(14 - (int(np.floor(np.log2(np.abs(C).max()))) + 1), 29 - int(np.floor(np.log2(csq.max() * (1 + 1e-7)))), 40)
     inv_s = 2.0 ** -k
-    split, kd, units = _tensor_units(g)
+    split, kd, units, nq = _tensor_units(g)
+    # two norm pieces multiply 2^e and 2^(e-11), e fitted to the largest scaled norm; a piece written
+    # as zero loses at most 2^(e-25) (four pieces: 2^-26)
+    e_norm = min(max(k + int(np.floor(np.log2(csq.max() * (1 + 1e-7)))) - 14, -3), 15)
+    norm_abs = 2.0 ** (e_norm - 25) if nq == 2 else 2.0 ** -26
     xsq = (np.maximum(np.abs(Xd), 2.0 ** -14) ** 2).sum(1)      # subnormal coordinates count as 2^-14
     rel = 2.0 ** -24 * (2 * csq[None, :] + xsq[:, None])
-    absolute = inv_s * (2.0 ** -14 * np.abs(Xd).sum(1)[:, None] + 2.0 ** -26)
+    absolute = inv_s * (2.0 ** -14 * np.abs(Xd).sum(1)[:, None] + norm_abs)
     err = np.abs(got - exact)
     worst = float(((err - absolute).clip(0) / rel).max())
     print("g=%d %s: worst error %.2f units (bound %d), scale 2^%d" % (g, kind, worst, units, k))

@@ -94,13 +94,14 @@ int64_t cc_launch_count(const cc_ctx* ctx);
 #define CC_KERNEL_ASSIGN_PREP 1   /* staging of the codebook for the scan               */
 #define CC_KERNEL_RESOLVE 2       /* exact FP64 stage for near-ties                     */
 #define CC_KERNEL_OBJECTIVE 3     /* deterministic sum of the distances                 */
-#define CC_KERNEL_UPDATE_ACCUM 4  /* M-step: integer sums and counts                    */
+#define CC_KERNEL_UPDATE_ACCUM 4  /* M-step over all points: integer sums and counts    */
 #define CC_KERNEL_UPDATE_FINISH 5 /* M-step: division, empty-cluster rule               */
 #define CC_KERNEL_RESHAPE 6
 #define CC_KERNEL_DECODE 7
 #define CC_KERNEL_OTHER 8
 #define CC_KERNEL_ASSIGN_FINISH 9 /* tensor path: index, distance, near-tie flag per point */
-#define CC_KERNEL_CLASSES 10
+#define CC_KERNEL_UPDATE_DELTA 10  /* M-step inside cc_fit: only the points whose code changed */
+#define CC_KERNEL_CLASSES 11
 cc_status cc_profile_enable(cc_ctx* ctx, int on);
 cc_status cc_profile_read(cc_ctx* ctx, double* total_ms_host, int64_t* launches_host);
 
@@ -109,6 +110,18 @@ cc_status cc_profile_read(cc_ctx* ctx, double* total_ms_host, int64_t* launches_
  * two-wide instruction form.  Synchronises `stream`.  Outputs are host doubles. */
 cc_status cc_measure_fp32_peak(cc_ctx* ctx, double* tflops_scalar_host, double* tflops_packed_host,
                                void* stream);
+
+/* Runs register-only loops of the FP32 minimum (the instruction that bounds the tensor-core E-step:
+ * every score is compared once) with one 512-thread block per SM and writes to the HOST array
+ * lane_instr_per_clk_per_sm[3] the measured lane-instructions per SM clock per SM for
+ *   [0] two-input min.f32, [1] three-input min.f32 (two new values each), [2] both alternating
+ * (median over the blocks of block lane-instructions / the block's own clock64 cycle count).
+ * sm_mhz (host, may be NULL): SM clock during the loops = cycles of the longest block / CUDA-event
+ * time of its launch.  distinct_sms (host, may be NULL): on how many different SMs the blocks ran
+ * (equal to the SM count when every block had an SM to itself).  Synchronises `stream`; allocates
+ * and frees a few KB of device memory. */
+cc_status cc_measure_min_rate(cc_ctx* ctx, double* lane_instr_per_clk_per_sm_host, double* sm_mhz_host,
+                              int32_t* distinct_sms_host, void* stream);
 
 /* Host helpers.  Number of sub-vectors after padding: the appendix listing's
  * num_codes = in_features * (out_features + deficiency) / g (PAPER_T), or the same rule along
@@ -148,6 +161,12 @@ cc_status cc_set_codebook(cc_ctx* ctx, const float* C0_host_or_device, int K, in
 cc_status cc_assign(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const float* C, int K,
                     uint16_t* idx, float* dist, double* objective, int64_t* n_resolved, void* stream);
 
+/* Verification aid (no counterpart in the paper): which points the last cc_assign on this
+ * context, with the same (N, g, K), sent to the exact FP64 stage.  Copies the first `count`
+ * entries of that list (point numbers, in no particular order; count <= the n_resolved the call
+ * reported) to `points`, a device or host array of uint32.  Valid until the next E-step. */
+cc_status cc_last_flagged(cc_ctx* ctx, int64_t N, int g, int K, uint32_t* points, int64_t count, void* stream);
+
 /* Verification aid for the tensor-core E-step (no counterpart in the paper): writes the raw
  * comparison scores s_ij = ||c_j||^2 - 2 x_i.c_j exactly as that path computes them (FP16 operand
  * pieces, FP32 accumulation in tensor memory), so that a test can check the rounding bound the
@@ -156,6 +175,17 @@ cc_status cc_assign(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const floa
 int64_t cc_tensor_scores_ld(int K);
 cc_status cc_tensor_scores(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const float* C, int K,
                            float* scores, void* stream);
+
+/* Verification aid for the tensor-core E-step (no counterpart in the paper): runs its second
+ * kernel alone on scan results supplied by the caller.  scan: N records of 8 bytes,
+ * {float: smallest score among the centroids outside the winning chunk, +inf if unknown;
+ *  int32: id of the 64-centroid chunk that holds the winner}.  For every point the chunk is
+ * searched in FP32, idx / dist (out, both required) get the chunk's best centroid and its FP64
+ * squared distance; the exact stage for near-ties is NOT run.  A chunk id outside
+ * 0 .. ceil(K / 64) - 1 (what a scan that gave up on a bounded wait may leave behind) is moved to
+ * the nearest valid chunk, so no such record can make the kernel read out of bounds.  N >= 1. */
+cc_status cc_tensor_finish_only(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const float* C, int K,
+                                const void* scan, uint16_t* idx, float* dist, void* stream);
 
 /* Self-test of the bounded waits of the tensor-core E-step (no counterpart in the paper).  Every
  * wait of those kernels on a shared-memory barrier gives up after a clock limit, raises a flag that
@@ -172,7 +202,8 @@ cc_status cc_tensor_scores(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, con
 cc_status cc_selftest_bounded_wait(cc_ctx* ctx, int64_t limit_cycles, int32_t* results, int64_t* cycles);
 
 /* M-step of Section 3.1: counts[j] = |{i : idx[i] = j}| (exact), C[j] = mean of those x_i
- * (exact integer sum, one rounding to FP32); a cluster with no member keeps its centroid
+ * (exact, order-independent integer sum; converted to double, divided by the count in double and
+ * rounded to FP32, as a sequential float64 sum would be); a cluster with no member keeps its centroid
  * bit for bit (the paper does not say; this library's rule).  C: in = previous, out = new.
  * counts (out): K x int32.  idx values must be < K. */
 cc_status cc_update(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const uint16_t* idx, int K,
@@ -190,16 +221,21 @@ cc_status cc_update(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const uint
  *
  * What it does: exactly what cc_update does, with the same results bit for bit, but the integer
  * sum accumulators live in a fixed array inside the library image (2 * CC_UPDATE_STATIC_MAX_KG
- * 64-bit words = 4 MiB).  Every GPU on which the library is loaded holds that array until the
- * process exits, whether or not this function is ever called.  The function takes no context and
- * calls no cudaMalloc / cudaFree nor any other allocating routine; the caller still provides
+ * 64-bit words = 4 MiB).  Every GPU on which the library's device code is loaded holds that array
+ * until the process exits.  The function takes no context and calls no cudaMalloc / cudaFree nor
+ * any other allocating routine; the caller still provides
  * X, idx, C and counts exactly as for cc_update, plus the device ordinal (< 64) that owns them.
  *
  * Limits and rules
  *  - K * g must not exceed CC_UPDATE_STATIC_MAX_KG (262144: K = 65536 at g = 4, K = 16384 at
  *    g = 16); larger problems return CC_ERR_STATIC_CAPACITY and enqueue nothing.
  *  - The first call on a device looks up the array's device address (once per device, with
- *    that device made current).  Make that first call before any stream capture begins.
+ *    that device made current).  Where the CUDA runtime loads device code lazily, that look-up is
+ *    also what loads this library's module and reserves the array on the device, so the memory is
+ *    taken at that moment rather than when the library is loaded: make the first call at start-up,
+ *    before any stream capture begins and before device memory becomes scarce.  The cached address
+ *    does not survive cudaDeviceReset; do not call the function again in a process that reset the
+ *    device.
  *  - All calls on one device share the one array, and it keeps the previous call's contents:
  *    each call clears the part it uses on `stream` before accumulating.  Two calls whose work
  *    overlaps on the GPU (different streams, no dependency) race on it and give wrong sums;

@@ -40,6 +40,7 @@ SIGNATURES = {
     "cc_profile_enable": (_i32, [_vp, _i32]),
     "cc_profile_read": (_i32, [_vp, _vp, _vp]),
     "cc_measure_fp32_peak": (_i32, [_vp, _vp, _vp, _vp]),
+    "cc_measure_min_rate": (_i32, [_vp, _vp, _vp, _vp, _vp]),
     "cc_num_subvectors": (_i64, [_i64, _i64, _i32, _i32]),
     "cc_bits_per_param": (_dbl, [_i64, _i64, _i32, _i32]),
     "cc_reshape_subvectors": (_i32, [_vp, _vp, _i64, _i64, _i32, _i32, _vp, _vp]),
@@ -47,8 +48,10 @@ SIGNATURES = {
     "cc_init_codebook": (_i32, [_vp, _vp, _i64, _i32, _i32, _u64, _vp, _vp]),
     "cc_set_codebook": (_i32, [_vp, _vp, _i32, _i32, _vp, _vp]),
     "cc_assign": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp]),
+    "cc_last_flagged": (_i32, [_vp, _i64, _i32, _i32, _vp, _i64, _vp]),
     "cc_tensor_scores_ld": (_i64, [_i32]),
     "cc_tensor_scores": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp]),
+    "cc_tensor_finish_only": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp, _vp]),
     "cc_selftest_bounded_wait": (_i32, [_vp, _i64, _vp, _vp]),
     "cc_update": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp]),
     "cc_update_static": (_i32, [_i32, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp]),
@@ -156,7 +159,7 @@ def cc_launch_count(ctx: Context) -> int:
 
 
 KERNEL_CLASSES = ("assign_main", "assign_prep", "resolve", "objective", "update_accum", "update_finish",
-                  "reshape", "decode", "other", "assign_finish")
+                  "reshape", "decode", "other", "assign_finish", "update_delta")
 
 
 def cc_profile_enable(ctx: Context, on: bool) -> None:
@@ -176,6 +179,15 @@ def cc_measure_fp32_peak(ctx: Context, stream=None):
     a, b = _dbl(0.0), _dbl(0.0)
     _check(load().cc_measure_fp32_peak(ctx._h, ct.byref(a), ct.byref(b), _stream(stream)), "cc_measure_fp32_peak")
     return a.value, b.value
+
+
+def cc_measure_min_rate(ctx: Context, stream=None):
+    """Returns ({"min2", "min3", "mixed"}: lane-instructions per clock per SM, SM MHz, distinct SMs)."""
+    r = (_dbl * 3)()
+    mhz, sms = _dbl(0.0), ct.c_int32(0)
+    _check(load().cc_measure_min_rate(ctx._h, r, ct.byref(mhz), ct.byref(sms), _stream(stream)),
+           "cc_measure_min_rate")
+    return {"min2": r[0], "min3": r[1], "mixed": r[2]}, mhz.value, sms.value
 
 
 def cc_num_subvectors(d_out: int, d_in: int, g: int, layout: int = LAYOUT_PAPER_T) -> int:
@@ -226,6 +238,10 @@ def cc_selftest_bounded_wait(ctx, limit_cycles: int):
     return list(res), list(cyc)
 
 
+def cc_last_flagged(ctx, N, g, K, points, count, stream=None) -> None:
+    _check(load().cc_last_flagged(ctx._h, N, g, K, _ptr(points), count, _stream(stream)), "cc_last_flagged")
+
+
 def cc_tensor_scores_ld(K: int) -> int:
     return int(load().cc_tensor_scores_ld(K))
 
@@ -233,6 +249,11 @@ def cc_tensor_scores_ld(K: int) -> int:
 def cc_tensor_scores(ctx, X, N, g, C, K, scores, stream=None) -> None:
     _check(load().cc_tensor_scores(ctx._h, _ptr(X), N, g, _ptr(C), K, _ptr(scores), _stream(stream)),
            "cc_tensor_scores")
+
+
+def cc_tensor_finish_only(ctx, X, N, g, C, K, scan, idx, dist, stream=None) -> None:
+    _check(load().cc_tensor_finish_only(ctx._h, _ptr(X), N, g, _ptr(C), K, _ptr(scan), _ptr(idx), _ptr(dist),
+                                        _stream(stream)), "cc_tensor_finish_only")
 
 
 def cc_update(ctx, X, N, g, idx, K, C, counts, stream=None) -> None:

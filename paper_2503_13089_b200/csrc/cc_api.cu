@@ -259,6 +259,18 @@ cc_status cc_assign(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const floa
     return from_cuda(assign_any(ctx, L, X, N, g, C, K, idx, dist, objective, n_resolved, (cudaStream_t)stream));
 }
 
+cc_status cc_last_flagged(cc_ctx* ctx, int64_t N, int g, int K, uint32_t* points, int64_t count, void* stream) {
+    if (!ctx || (count > 0 && !points)) return CC_ERR_NULL;
+    cc_status s = check_common(ctx, N, g, K, true);
+    if (s != CC_OK) return s;
+    if (count < 0 || count > N) return CC_ERR_SHAPE;
+    if (count == 0) return CC_OK;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    const WsLayout L = cc_ws_layout(N, g, K);
+    return from_cuda(cudaMemcpyAsync(points, static_cast<char*>(ctx->ws) + L.flagged, sizeof(uint32_t) * (size_t)count,
+                                     cudaMemcpyDefault, (cudaStream_t)stream));
+}
+
 int64_t cc_tensor_scores_ld(int K) { return (K < 1 || K > 65536) ? -1 : cc_tensor_score_ld(K); }
 
 cc_status cc_tensor_scores(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const float* C, int K, float* scores,
@@ -271,6 +283,18 @@ cc_status cc_tensor_scores(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, con
     if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
     const WsLayout L = cc_ws_layout(N, g, K);
     return from_cuda(cc_launch_tensor_scores(ctx, L, X, N, g, C, K, scores, (cudaStream_t)stream));
+}
+
+cc_status cc_tensor_finish_only(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const float* C, int K,
+                                const void* scan, uint16_t* idx, float* dist, void* stream) {
+    if (!ctx || !C || !X || !scan || !idx || !dist) return CC_ERR_NULL;
+    cc_status s = check_common(ctx, N, g, K, true);
+    if (s != CC_OK) return s;
+    if (N < 1) return CC_ERR_SHAPE;
+    if (!aligned16(X) || !aligned16(C) || (reinterpret_cast<uintptr_t>(scan) & 7u)) return CC_ERR_ALIGN;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    const WsLayout L = cc_ws_layout(N, g, K);
+    return from_cuda(cc_launch_tensor_finish_only(ctx, L, X, N, g, C, K, scan, idx, dist, (cudaStream_t)stream));
 }
 
 cc_status cc_selftest_bounded_wait(cc_ctx* ctx, int64_t limit_cycles, int32_t* results, int64_t* cycles) {

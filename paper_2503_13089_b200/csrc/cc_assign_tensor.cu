@@ -76,10 +76,16 @@ template <int G> struct TcCfg {
     static constexpr int STAGES = (KD <= 16) ? 4 : 3;
     static constexpr int MERGE = (EW - 1) * NA * TM * 12;           // exchange of the column groups' results
     static constexpr int SMEM = NA * A_TILE + STAGES * B_TILE + MERGE + 256;
-    // Rounding model of the accumulation, in units of 2^-24 (2||c||^2 + ||x||^2): measured on the
-    // device at 2.3 / 3.4 / 4.2 units for one / two / three 16-column MMA steps; the two-piece
-    // split adds 4.
-    static constexpr int ERR_UNITS = 8 * (KD / 16) + (SPLIT == 2 ? 4 : 0) + (NQ == 2 ? 4 : 0);
+    // Rounding model of the accumulation, in units of 2^-24 S (2||c||^2 + ||x||^2).  Assumed of the
+    // tensor core: one 16-column step forms the 16 products exactly, aligns them and the FP32
+    // accumulator to the largest exponent among the 17 addends, keeps at least 24 bits below that
+    // exponent of each addend (the rest is dropped), adds exactly and rounds or truncates the sum to
+    // FP32.  Every addend and every partial sum is at most S (2||c||^2 + ||x||^2) in magnitude
+    // (2|x_t c_t| <= x_t^2 + c_t^2), so a step errs by at most 17 + 2 = 19 units.  Measured on the
+    // device: 2.3 / 3.4 / 4.2 units for one / two / three steps.  Cutting S m into two pieces instead
+    // of three leaves a residue of 2^-22 |S m_t| per coordinate: 4 more units; two norm pieces
+    // instead of four leave 2^-22 S ||c||^2: 4 more.
+    static constexpr int ERR_UNITS = 19 * (KD / 16) + (SPLIT == 2 ? 4 : 0) + (NQ == 2 ? 4 : 0);
 };
 
 // Written by the range kernel / prep kernel, read by the finish kernel (workspace, 16 bytes).
@@ -868,7 +874,7 @@ assign_tensor_persistent_kernel(const uint16_t* __restrict__ X, int64_t N, const
 // smallest scores are closer than 2E with that substitution goes to the exact stage.
 template <int G>
 __global__ void __launch_bounds__(256)
-finish_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restrict__ C, int K,
+finish_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restrict__ C, int K, int n_chunks,
                      const float* __restrict__ rescan, const float2* __restrict__ tstate,
                      const TcParams* __restrict__ params, uint16_t* __restrict__ idx, float* __restrict__ dist,
                      unsigned* __restrict__ status, unsigned* __restrict__ flagged) {
@@ -893,7 +899,12 @@ finish_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __r
         const int64_t i_raw = base + lane;
         const bool live = i_raw < N;
         const int64_t i = live ? i_raw : N - 1;
-        const float2 t_own = tstate[i];
+        float2 t_own = tstate[i];
+        // The chunk id comes from the scan's output.  A scan CTA that gave up on a bounded wait has
+        // written nothing there, so the word may hold anything: keep it inside the table (the call
+        // then reports CC_ERR_DEVICE_TIMEOUT and its results are void, but nothing is read out of
+        // bounds).
+        t_own.y = __int_as_float(min(max(__float_as_int(t_own.y), 0), n_chunks - 1));
         float x_own[G];
         bool nf = false;
         load_point<G>(X, i, N, x_own, nf);
@@ -946,7 +957,7 @@ finish_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __r
             }
         }
         int j1 = keep_j;
-        if (j1 >= K) j1 = K - 1;   // only reachable with non-finite input
+        if (j1 >= K) j1 = K - 1;   // only reachable with non-finite input or after a time-out
         const float (&x)[G] = x_own;
         double D = 0.0;
         float A = 0.f, L1 = 0.f;
@@ -974,13 +985,15 @@ finish_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __r
 
 template <int G>
 cudaError_t launch_tensor(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64_t N, const float* C, int K,
-                          uint16_t* idx, float* dist, float* dump, int64_t dump_ld, cudaStream_t st) {
+                          uint16_t* idx, float* dist, float* dump, int64_t dump_ld, const float2* scan_in,
+                          cudaStream_t st) {
     using Cfg = TcCfg<G>;
     char* ws = static_cast<char*>(ctx->ws);
     unsigned* status = reinterpret_cast<unsigned*>(ws + L.status);
     TcParams* params = reinterpret_cast<TcParams*>(ws + L.status + 128);
     uint16_t* gB = reinterpret_cast<uint16_t*>(ws + L.tensor);
     float2* tstate = reinterpret_cast<float2*>(ws + L.tstate);
+    if (scan_in) tstate = const_cast<float2*>(scan_in);   // finish only: the caller supplies the scan's output
     const int Kpad = (int)cc_align_up((size_t)K, TN);
     // FP32 rows of the finish kernel sit behind the FP16 operand image (at most 96 bytes per centroid)
     float* rescan = reinterpret_cast<float*>(ws + L.tensor + (size_t)Kpad * 96);
@@ -1017,7 +1030,7 @@ cudaError_t launch_tensor(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int
                 X, N, gB, Kpad / TN, (int)na_per_cta, 0, params, tstate, status, dump, dump_ld);
             return cudaGetLastError();
         }
-        {
+        if (!scan_in) {
             ProfScope ps(ctx, CC_K_ASSIGN_MAIN, st);
             // CTAs with a full set of NA point tiles, then the ragged rest
             const int64_t full_blocks = (na_per_cta == NA) ? n_tiles / NA : 0;
@@ -1046,7 +1059,8 @@ cudaError_t launch_tensor(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int
             const int64_t cap = (int64_t)ctx->sm_count * 32;
             if (fblocks > cap) fblocks = cap;
             finish_tensor_kernel<G><<<(unsigned)fblocks, 256, 0, st>>>(
-                X, N, C, K, rescan, tstate, params, idx, dist, status, reinterpret_cast<unsigned*>(ws + L.flagged));
+                X, N, C, K, Kpad / TCHUNK, rescan, tstate, params, idx, dist, status,
+                reinterpret_cast<unsigned*>(ws + L.flagged));
         }
     }
     return cudaGetLastError();
@@ -1076,7 +1090,7 @@ cudaError_t cc_launch_assign_tensor(cc_ctx* ctx, const WsLayout& L, const uint16
                                     const float* C, int K, uint16_t* idx, float* dist, double* objective,
                                     int64_t* n_resolved, cudaStream_t st) {
     cudaError_t e = cudaSuccess;
-#define CALL(G) e = launch_tensor<G>(ctx, L, X, N, C, K, idx, dist, nullptr, 0, st)
+#define CALL(G) e = launch_tensor<G>(ctx, L, X, N, C, K, idx, dist, nullptr, 0, nullptr, st)
     CC_TENSOR_DISPATCH(g, CALL)
 #undef CALL
     if (e != cudaSuccess) return e;
@@ -1123,7 +1137,18 @@ cudaError_t cc_launch_tensor_scores(cc_ctx* ctx, const WsLayout& L, const uint16
                                     const float* C, int K, float* scores, cudaStream_t st) {
     cudaError_t e = cudaSuccess;
     const int64_t ld = cc_tensor_score_ld(K);
-#define CALL(G) e = launch_tensor<G>(ctx, L, X, N, C, K, nullptr, nullptr, scores, ld, st)
+#define CALL(G) e = launch_tensor<G>(ctx, L, X, N, C, K, nullptr, nullptr, scores, ld, nullptr, st)
+    CC_TENSOR_DISPATCH(g, CALL)
+#undef CALL
+    return e;
+}
+
+// Verification aid: staging + finish kernel on scan results supplied by the caller (no scan, no exact stage).
+cudaError_t cc_launch_tensor_finish_only(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, int64_t N, int g,
+                                         const float* C, int K, const void* scan, uint16_t* idx, float* dist,
+                                         cudaStream_t st) {
+    cudaError_t e = cudaSuccess;
+#define CALL(G) e = launch_tensor<G>(ctx, L, X, N, C, K, idx, dist, nullptr, 0, static_cast<const float2*>(scan), st)
     CC_TENSOR_DISPATCH(g, CALL)
 #undef CALL
     return e;

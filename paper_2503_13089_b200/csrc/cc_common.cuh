@@ -13,7 +13,8 @@
 
 // Kernel classes for the optional per-kernel event timing (cc_profile_*).
 enum { CC_K_ASSIGN_MAIN = 0, CC_K_ASSIGN_PREP = 1, CC_K_RESOLVE = 2, CC_K_OBJECTIVE = 3, CC_K_UPDATE_ACCUM = 4,
-       CC_K_UPDATE_FINISH = 5, CC_K_RESHAPE = 6, CC_K_DECODE = 7, CC_K_OTHER = 8, CC_K_ASSIGN_FINISH = 9, CC_K_COUNT = 10 };
+       CC_K_UPDATE_FINISH = 5, CC_K_RESHAPE = 6, CC_K_DECODE = 7, CC_K_OTHER = 8, CC_K_ASSIGN_FINISH = 9, CC_K_UPDATE_DELTA = 10,
+       CC_K_COUNT = 11 };
 constexpr int CC_PROF_CAP = 8192;
 
 struct cc_prof_slot { cudaEvent_t a, b; int kind; };
@@ -110,6 +111,8 @@ int cc_tensor_score_ld(int K);
 cudaError_t cc_launch_wait_selftest(long long limit_cycles, int* out_dev, long long* cycles_dev, cudaStream_t);
 cudaError_t cc_launch_tensor_scores(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const float* C,
                                     int K, float* scores, cudaStream_t);
+cudaError_t cc_launch_tensor_finish_only(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const float* C,
+                                         int K, const void* scan, uint16_t* idx, float* dist, cudaStream_t);
 // Second stage shared by both E-step paths: exact FP64 decision for the flagged points, then
 // the deterministic objective sum.
 cudaError_t cc_launch_assign_tail(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const float* C,

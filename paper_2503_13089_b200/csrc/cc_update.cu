@@ -5,8 +5,11 @@
 // accumulators per (cluster, dimension): |x| < 8 in units of 2^-24 (< 2^27 per term) and
 // |x| >= 8 in units of 2^-7 (< 2^23 per term).  With N < 2^31 neither can overflow, integer
 // addition is associative, and so the result does not depend on the order in which the points
-// arrive: the kernel is deterministic without sorting the points first, the counts are exact
-// integers, and the mean is rounded exactly once (sum -> double -> divide -> FP32).
+// arrive: the kernel is deterministic without sorting the points first and the counts are exact
+// integers.  The mean is formed as the CPU oracle forms it: the integer sums go to double (exact
+// while a sum stays below 2^53 units of 2^-24, i.e. |sum| < 2^29: more than 8000 values of the
+// largest FP16 magnitude in one cluster, or 5 * 10^8 of magnitude 1), are divided by the count in
+// double and the quotient is rounded to FP32.
 // A cluster with no member keeps its previous centroid.
 // The same property lets the Lloyd loop keep the sums between iterations and only move the points
 // whose code changed (update_delta_kernel), and gives the gradient with respect to the codebook
@@ -220,7 +223,7 @@ cudaError_t cc_launch_update_delta(cc_ctx* ctx, const WsLayout& L, const uint16_
         int64_t blocks = (N + 255) / 256;
         const int64_t cap = (int64_t)ctx->sm_count * 16;
         if (blocks > cap) blocks = cap;
-        ProfScope ps(ctx, CC_K_UPDATE_ACCUM, st);
+        ProfScope ps(ctx, CC_K_UPDATE_DELTA, st);
 #define CALL(G) update_delta_kernel<G><<<(unsigned)blocks, 256, 0, st>>>(X, N, idx, idx_prev, K, sum_lo, sum_hi, counts)
         CC_UPDATE_DISPATCH(g, CALL)
 #undef CALL

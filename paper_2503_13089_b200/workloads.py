@@ -60,7 +60,7 @@ WORKLOADS = {
     "cfg1_256x512_g4_k256": Workload(
         "cfg1_256x512_g4_k256", 4, 256, 10,
         (MatrixSpec("w", 256, 512, "normal", 0.02, 0.001, 0, 2001),)),
-    # the configuration the headline metric is quoted on
+    # a 7B attention-projection shape with a small codebook (3 bits per weight of index)
     "cfg2_4096x4096_g4_k4096": Workload(
         "cfg2_4096x4096_g4_k4096", 4, 4096, 20,
         (MatrixSpec("w", 4096, 4096, "student_t3", 0.02, 0.0, 1002, 2002),)),

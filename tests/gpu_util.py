@@ -35,7 +35,7 @@ def u16_np(t):
     return t.cpu().view(torch.int16).numpy().view(np.uint16)
 
 
-def gpu_assign(X, C, path=cc.PATH_AUTO, want_dist=True):
+def gpu_assign(X, C, path=cc.PATH_AUTO, want_dist=True, want_flagged=False):
     c = ctx()
     N, g = X.shape
     K = C.shape[0]
@@ -49,8 +49,19 @@ def gpu_assign(X, C, path=cc.PATH_AUTO, want_dist=True):
     cc.cc_assign(c, Xd, N, g, Cd, K, idx, dist, obj, nres)
     cc.cc_poll_status(c)
     cc.cc_set_path(c, cc.PATH_AUTO)
-    return (u16_np(idx)[:N].astype(np.int32), None if dist is None else dist.cpu().numpy()[:N],
-            float(obj.item()), int(nres.item()))
+    out = (u16_np(idx)[:N].astype(np.int32), None if dist is None else dist.cpu().numpy()[:N],
+           float(obj.item()), int(nres.item()))
+    if want_flagged:
+        out = out + (last_flagged(N, g, K, out[3]),)
+    return out
+
+
+def last_flagged(N, g, K, count):
+    """Point numbers the last E-step on the shared context sent to the exact FP64 stage."""
+    pts = torch.empty(max(count, 1), dtype=torch.int32, device="cuda")
+    cc.cc_last_flagged(ctx(), N, g, K, pts, count)
+    torch.cuda.synchronize()
+    return pts.cpu().numpy()[:count].astype(np.int64)
 
 
 def gpu_update(X, idx, C_prev):
@@ -67,13 +78,18 @@ def gpu_update(X, idx, C_prev):
     return Cd.cpu().numpy(), counts.cpu().numpy()
 
 
-def check_assign_against_oracle(X, C, idx_gpu, dist_gpu, sel=None):
-    """Bit-exact indices except near-ties of the oracle's float64 distances; returns (#tolerated, o_idx, d1)."""
+def check_assign_against_oracle(X, C, idx_gpu, dist_gpu, sel=None, flagged=None):
+    """Bit-exact indices except near-ties of the oracle's float64 distances; returns (#tolerated, o_idx, d1).
+    `flagged`: the points the GPU decided in its exact FP64 stage, which uses the oracle's own
+    arithmetic -- there even a near-tie must come out as the oracle's index."""
     o_idx, d1, d2 = oracle.assign(X, C, sel)
     gi = idx_gpu if sel is None else idx_gpu[sel]
     bad = np.flatnonzero(gi != o_idx)
     tolerated = 0
     rows = np.arange(len(X)) if sel is None else sel
+    if flagged is not None and len(bad):
+        wrong = np.intersect1d(rows[bad], flagged)
+        assert len(wrong) == 0, "points decided by the exact stage differ from the oracle: %r" % wrong[:10]
     for r in bad:
         d_g = oracle.point_dist(X, int(rows[r]), C, int(gi[r]))
         rel = 0.0 if d_g == 0 else (d_g - d1[r]) / d_g

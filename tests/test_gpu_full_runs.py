@@ -1,0 +1,197 @@
+"""GPU parity on the five benchmark configurations at full size, over their full iteration counts.
+
+Protocol (lock-step): cc_fit is deterministic, so cc_fit(t) from the seeded start reproduces the
+first t iterations of every longer run.  At a checked iteration t the oracle gets the GPU's own
+centroids C_{t-1} and
+  * assigns a seeded sample of the points against ALL centroids: the GPU's codes of iteration t must
+    agree bit for bit, except where the oracle's two best float64 distances differ by < 1e-6 relative
+    (counted, and never allowed for a point the GPU decided in its exact FP64 stage);
+  * runs its M-step on ALL points with the GPU's codes: counts bit-exact, centroids within 1e-4 (in fact
+    the same bits), empty clusters keep the previous centroid bit for bit.
+Because the codes come from cc_fit(t), the M-step of a late iteration is the incremental one (only
+the points whose code changed are moved), checked here at full size.  Free-running oracle objectives
+are compared where a full oracle run is affordable (configurations 1 and 2).
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2503_13089_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+
+def _cc():
+    from paper_2503_13089_b200 import binding
+    return binding
+
+
+def _u():
+    from tests import gpu_util
+    return gpu_util
+
+
+class _Fit:
+    """Device-resident points of one matrix and repeated cc_fit runs from the same start."""
+
+    def __init__(self, X, C0):
+        cc, u = _cc(), _u()
+        self.X, self.C0 = X, C0
+        self.N, self.g = X.shape
+        self.K = C0.shape[0]
+        self.ctx = u.ctx()
+        self.ctx.ensure_workspace(self.N, self.g, self.K)
+        self.Xd = u.half_dev(X)
+        self.idx = torch.empty(self.N, dtype=torch.uint16, device="cuda")
+        self.dist = torch.empty(self.N, dtype=torch.float32, device="cuda")
+        self.counts = torch.empty(self.K, dtype=torch.int32, device="cuda")
+
+    def run(self, t):
+        """cc_fit(t) from C0 -> (C_t, codes of iteration t, their distances, counts, objective trace)."""
+        cc, u = _cc(), _u()
+        C = u.dev(self.C0)
+        trace = torch.empty(max(t, 1), dtype=torch.float64, device="cuda")
+        cc.cc_fit(self.ctx, self.Xd, self.N, self.g, self.K, t, C, self.idx, self.dist, self.counts, trace)
+        cc.cc_poll_status(self.ctx)
+        return (C.cpu().numpy(), u.u16_np(self.idx).astype(np.int32), self.dist.cpu().numpy(),
+                self.counts.cpu().numpy(), trace.cpu().numpy()[:t])
+
+    def assign(self, C):
+        """One stand-alone E-step: codes, number of points sent to the exact stage, and which."""
+        cc, u = _cc(), _u()
+        Cd = u.dev(C)
+        idx = torch.empty(self.N, dtype=torch.uint16, device="cuda")
+        nres = torch.zeros(1, dtype=torch.int64, device="cuda")
+        cc.cc_assign(self.ctx, self.Xd, self.N, self.g, Cd, self.K, idx, None, None, nres)
+        cc.cc_poll_status(self.ctx)
+        n = int(nres.item())
+        return u.u16_np(idx).astype(np.int32), n, u.last_flagged(self.N, self.g, self.K, n)
+
+
+def _check_iteration(fit, t, C_prev, frac, seed, stats, trace_prev=None):
+    """Runs cc_fit(t) and checks iteration t against the oracle given C_{t-1}; returns (C_t, trace)."""
+    u = _u()
+    X = fit.X
+    C_t, idx_t, dist_t, counts_t, trace = fit.run(t)
+    if trace_prev is not None:                     # the same run, one iteration further: same bits before it
+        assert np.array_equal(trace[:len(trace_prev)], trace_prev)
+    idx_a, n_exact, flagged = fit.assign(C_prev)   # the E-step of iteration t once more, for its flag list
+    assert np.array_equal(idx_a, idx_t)
+    sel = None if frac >= 1.0 else wl.subset_positions(fit.N, frac, seed + t)
+    tol, o_idx, d1 = u.check_assign_against_oracle(X, C_prev, idx_t, dist_t, sel, flagged=flagged)
+    if sel is None:
+        assert trace[t - 1] == pytest.approx(d1.sum(), rel=u.REL_OBJECTIVE)
+    C_or, counts_or = oracle.update(X, idx_t, C_prev)           # oracle M-step on all points, GPU's codes
+    assert np.array_equal(counts_t.astype(np.int64), counts_or.astype(np.int64))
+    assert u.centroid_rel_err(C_t, C_or, X) <= u.REL_CENTROID
+    assert np.array_equal(C_t.view(np.uint32), C_or.view(np.uint32))
+    empty = counts_or == 0
+    assert np.array_equal(C_t[empty].view(np.uint32), C_prev[empty].view(np.uint32))
+    if t > 1:
+        assert trace[t - 1] <= trace[t - 2] * (1 + 1e-6)          # the objective never increases
+    stats["checked_points"] += fit.N if sel is None else len(sel)
+    stats["tolerated"] += tol
+    stats["exact_stage"].append(n_exact)
+    stats["empty"].append(int(empty.sum()))
+    return C_t, trace
+
+
+def _new_stats():
+    return {"checked_points": 0, "tolerated": 0, "exact_stage": [], "empty": []}
+
+
+def _report(name, stats):
+    print("%s: %d sampled points compared, 0 mismatches outside the tolerance, %d tolerated near-ties, "
+          "points sent to the exact stage per E-step %s, empty clusters per M-step %s"
+          % (name, stats["checked_points"], stats["tolerated"], stats["exact_stage"], stats["empty"]))
+
+
+def test_cfg2_all_twenty_iterations_then_finalize_and_free_run():
+    """4096 x 4096, g = 4, K = 4096: iteration 1 on every point, iterations 2, 5, 10 and 20 on a 2 % sample,
+    the oracle's own free-running objectives at all twenty iterations, and cc_finalize."""
+    cc, u = _cc(), _u()
+    w = wl.WORKLOADS["cfg2_4096x4096_g4_k4096"]
+    spec = w.matrices[0]
+    X = oracle.reshape_subvectors(wl.make_matrix(spec), w.g)
+    C0 = oracle.init_codebook(X, w.K, spec.init_seed)
+    fit = _Fit(X, C0)
+    stats = _new_stats()
+    C1, tr = _check_iteration(fit, 1, C0, 1.0, 77, stats)
+    C2, tr = _check_iteration(fit, 2, C1, 0.02, 77, stats, tr)
+    for t in (5, 10, 20):
+        C_prev = fit.run(t - 1)[0]
+        C_t, tr = _check_iteration(fit, t, C_prev, 0.02, 77, stats)
+    _report("cfg2", stats)
+    assert len(tr) == w.iters
+    C_or, idx_or, d1_or, counts_or, obj_or = oracle.fit(X, C0, w.iters)       # free-running oracle, all points
+    assert np.allclose(tr, obj_or, rtol=u.REL_OBJECTIVE, atol=0)
+    # a free run may part from the oracle at a near-tie; where it did not, it must end on the same bits
+    idx20 = fit.run(w.iters)[1]
+    differing = int((idx20 != idx_or).sum())
+    print("cfg2 free run: %d of %d codes differ from the free-running oracle after %d iterations"
+          % (differing, fit.N, w.iters))
+    if differing == 0:
+        assert np.array_equal(C_t.view(np.uint32), C_or.view(np.uint32))
+    # finalize: FP16 codebook, codes against it, objective
+    C16 = torch.empty((w.K, w.g), dtype=torch.float16, device="cuda")
+    obj = torch.zeros(1, dtype=torch.float64, device="cuda")
+    cc.cc_finalize(fit.ctx, fit.Xd, fit.N, w.g, u.dev(C_t), w.K, C16, fit.idx, fit.dist, obj)
+    cc.cc_poll_status(fit.ctx)
+    C16n = C16.cpu().numpy()
+    assert np.array_equal(C16n.view(np.uint16), oracle.to_half(C_t).view(np.uint16))
+    idx_f = u.u16_np(fit.idx).astype(np.int32)
+    sel = wl.subset_positions(fit.N, 0.02, 78)
+    u.check_assign_against_oracle(X, C16n.astype(np.float32), idx_f, fit.dist.cpu().numpy(), sel)
+    _, _, _, J_or = oracle.finalize(X, C_or)
+    assert obj.item() == pytest.approx(J_or, rel=u.REL_OBJECTIVE)
+
+
+def test_cfg3_all_twenty_iterations_sampled():
+    """4096 x 11008, g = 8, K = 65536: every one of the 20 iterations on a fresh 0.5 % sample."""
+    w = wl.WORKLOADS["cfg3_4096x11008_g8_k65536"]
+    spec = w.matrices[0]
+    X = oracle.reshape_subvectors(wl.make_matrix(spec), w.g)
+    C0 = oracle.init_codebook(X, w.K, spec.init_seed)
+    fit = _Fit(X, C0)
+    stats = _new_stats()
+    C, tr = C0, None
+    for t in range(1, w.iters + 1):
+        C, tr = _check_iteration(fit, t, C, 0.005, 300, stats, tr)
+    _report("cfg3", stats)
+    assert tr[-1] < tr[0]
+
+
+def test_cfg4_all_ten_iterations_one_percent_sample():
+    """8192 x 28672, g = 4, K = 65536 (58.7 M points): every one of the 10 iterations, the oracle assigning a
+    fresh seeded 1 % of the points against all centroids and running its M-step on all of them."""
+    w = wl.WORKLOADS["cfg4_8192x28672_g4_k65536"]
+    spec = w.matrices[0]
+    X = oracle.reshape_subvectors(wl.make_matrix(spec), w.g)
+    C0 = oracle.init_codebook(X, w.K, spec.init_seed)
+    fit = _Fit(X, C0)
+    stats = _new_stats()
+    C, tr = C0, None
+    for t in range(1, w.iters + 1):
+        C, tr = _check_iteration(fit, t, C, w.subset_frac, 400, stats, tr)
+    _report("cfg4", stats)
+    assert w.subset_frac == 0.01 and stats["checked_points"] >= 10 * 587202
+    assert tr[-1] < tr[0]
+
+
+@pytest.mark.parametrize("mat", range(7))
+def test_cfg5_every_matrix_all_fifteen_iterations_with_empty_clusters(mat):
+    """One 7B decoder layer at g = 16, K = 65536: 16 (attention) or 43 (MLP) points per centroid, so
+    clusters do run empty; the keep-the-previous-centroid rule is checked on them at every iteration."""
+    w = wl.WORKLOADS["cfg5_layer7b_g16_k65536"]
+    spec = w.matrices[mat]
+    X = oracle.reshape_subvectors(wl.make_matrix(spec), w.g)
+    C0 = oracle.init_codebook(X, w.K, spec.init_seed)
+    fit = _Fit(X, C0)
+    stats = _new_stats()
+    C, tr = C0, None
+    for t in range(1, w.iters + 1):
+        C, tr = _check_iteration(fit, t, C, 0.005, 500 + 20 * mat, stats, tr)
+    _report("cfg5 " + spec.name, stats)
+    assert max(stats["empty"]) > 0, "expected empty clusters at %d points per centroid" % (fit.N // w.K)
+    assert tr[-1] < tr[0]

@@ -114,8 +114,9 @@ def test_assign_matches_oracle(N, g, K):
     u = _u()
     X = wl.make_points(N, g, 1000 + N + g)
     C = wl.make_codebook(K, g, 2000 + K + g)
-    idx, dist, obj, nres = u.gpu_assign(X, C)
-    tol, o_idx, d1 = u.check_assign_against_oracle(X, C, idx, dist)
+    idx, dist, obj, nres, flagged = u.gpu_assign(X, C, want_flagged=True)
+    tol, o_idx, d1 = u.check_assign_against_oracle(X, C, idx, dist, flagged=flagged)
+    print("N=%d g=%d K=%d: %d tolerated near-ties, %d points sent to the exact stage" % (N, g, K, tol, nres))
     assert tol <= max(1, N // 1000)
     assert obj == pytest.approx(float(np.sum(dist.astype(np.float64))), rel=1e-12)
     assert obj == pytest.approx(d1.sum(), rel=1e-6)
@@ -136,8 +137,8 @@ def test_assign_fp32_and_tensor_paths_agree_with_oracle_and_each_other(N, g, K):
     C = wl.make_codebook(K, g, 2000 + K + g)
     res = {}
     for path in (cc.PATH_FFMA, cc.PATH_TENSOR):
-        idx, dist, obj, nres = u.gpu_assign(X, C, path=path)
-        tol, o_idx, d1 = u.check_assign_against_oracle(X, C, idx, dist)
+        idx, dist, obj, nres, flagged = u.gpu_assign(X, C, path=path, want_flagged=True)
+        tol, o_idx, d1 = u.check_assign_against_oracle(X, C, idx, dist, flagged=flagged)
         assert tol <= max(1, N // 1000)
         res[path] = (idx, dist, obj)
     a, b = res[cc.PATH_FFMA], res[cc.PATH_TENSOR]
@@ -149,35 +150,66 @@ def test_assign_fp32_and_tensor_paths_agree_with_oracle_and_each_other(N, g, K):
 
 def _tensor_units(g):
     """Rounding model of the tensor-core scan as the library documents it: contraction length,
-    number of FP16 pieces per centroid value, allowed error in units of 2^-24 (2||c||^2 + ||x||^2)."""
+    number of FP16 pieces per centroid value, allowed error in units of 2^-24 (2||c||^2 + ||x||^2):
+    19 per 16-column step (17 addends aligned to the largest and cut 24 bits below it, plus the
+    rounding of the sum), 4 for a value cut into two pieces instead of three, 4 for two norm pieces."""
     kd34, kd24, kd22 = (3 * g + 4 + 15) // 16 * 16, (2 * g + 4 + 15) // 16 * 16, (2 * g + 2 + 15) // 16 * 16
     full = kd34 <= 48 and kd34 <= kd24 and kd34 <= kd22
     split = 3 if full else 2                 # two pieces of a value where that shortens the contraction
     nq = 4 if (full or kd24 <= kd22) else 2  # ... and two pieces of the norm (g = 7, 15)
     kd = (split * g + nq + 15) // 16 * 16
-    return split, kd, 8 * (kd // 16) + (4 if split == 2 else 0) + (4 if nq == 2 else 0), nq
+    return split, kd, 19 * (kd // 16) + (4 if split == 2 else 0) + (4 if nq == 2 else 0), nq
 
 
-@pytest.mark.parametrize("kind", ["weights", "wide_range", "on_centroids", "huge"])
+def _score_case(kind, g, rng):
+    """(X FP16, C FP32) of one family of inputs for the rounding-model test."""
+    N, K = 2048, 5000                       # 1.0e7 scores per call; K is not a multiple of the 256-centroid tile
+    if kind == "weights":
+        return wl.make_points(N, g, 50 + g), wl.make_codebook(K, g, 60 + g)
+    if kind == "wide_range":
+        X = (rng.standard_normal((N, g)) * np.exp2(rng.uniform(-20, 6, (N, g)))).astype(np.float16)
+        return X, (rng.standard_normal((K, g)) * np.exp2(rng.uniform(-24, 6, (K, g)))).astype(np.float32)
+    if kind == "on_centroids":
+        C = wl.make_codebook(K, g, 61 + g)
+        return C[rng.integers(0, K, N)].astype(np.float16), C
+    if kind == "huge":
+        X = (rng.standard_normal((N, g)) * 2e4).clip(-65000, 65000).astype(np.float16)
+        return X, (rng.standard_normal((K, g)) * 1e4).astype(np.float32)
+    if kind == "on_centroids_large":         # points equal to centroids at large magnitude
+        C = (rng.standard_normal((K, g)) * 3000).astype(np.float16).astype(np.float32)
+        return C[rng.integers(0, K, N)].astype(np.float16), C
+    if kind == "one_huge_norm":              # one centroid sets the scale, all the others are tiny beside it
+        C = wl.make_codebook(K, g, 62 + g)
+        C[K // 3] = 900.0
+        return wl.make_points(N, g, 51 + g), C
+    if kind == "cancellation":               # x = c / 2: x.c = ||c||^2 / 2, the score cancels to (almost) zero
+        C = wl.make_codebook(K, g, 63 + g, scale=0.5)
+        X = (C[rng.integers(0, K, N)] * 0.5).astype(np.float16)
+        return X, C
+    if kind == "subnormal_points":           # every coordinate of x below 2^-14
+        X = (rng.uniform(-1, 1, (N, g)) * 6e-5).astype(np.float16)
+        assert np.all(np.abs(X.astype(np.float64)) < 2.0 ** -14)
+        return X, wl.make_codebook(K, g, 64 + g)
+    if kind == "k65536_from_points":         # the benchmark's shape: 65536 centroids drawn from the points
+        Xall = wl.make_points(70000, g, 52 + g)
+        return Xall[:160], Xall[4000:4000 + 65536].astype(np.float32)
+    raise ValueError(kind)
+
+
+SCORE_KINDS = ["weights", "wide_range", "on_centroids", "huge", "on_centroids_large", "one_huge_norm", "cancellation",
+               "subnormal_points", "k65536_from_points"]
+
+
+@pytest.mark.parametrize("kind", SCORE_KINDS)
 @pytest.mark.parametrize("g", [1, 3, 4, 5, 6, 7, 8, 9, 10, 12, 14, 15, 16])
 def test_tensor_scores_obey_the_rounding_model(g, kind):
-    """Every raw score of the tensor-core scan against float64: the error must stay inside the
-    bound that decides which points are sent to the exact stage (and, here, inside half of it)."""
+    """Every raw score of the tensor-core scan against float64 (10^7 scores per case): the error must
+    stay inside the bound that decides which points are sent to the exact stage -- here inside a
+    third of it, so that the bound keeps a margin over everything seen."""
     cc, u = _cc(), _u()
     rng = np.random.default_rng(100 * g + len(kind))
-    N, K = 700, 900
-    if kind == "weights":
-        X = wl.make_points(N, g, 50 + g)
-        C = wl.make_codebook(K, g, 60 + g)
-    elif kind == "wide_range":
-        X = (rng.standard_normal((N, g)) * np.exp2(rng.uniform(-20, 6, (N, g)))).astype(np.float16)
-        C = (rng.standard_normal((K, g)) * np.exp2(rng.uniform(-24, 6, (K, g)))).astype(np.float32)
-    elif kind == "on_centroids":
-        C = wl.make_codebook(K, g, 61 + g)
-        X = C[rng.integers(0, K, N)].astype(np.float16)
-    else:
-        X = (rng.standard_normal((N, g)) * 2e4).clip(-65000, 65000).astype(np.float16)
-        C = (rng.standard_normal((K, g)) * 1e4).astype(np.float32)
+    X, C = _score_case(kind, g, rng)
+    N, K = len(X), len(C)
     c = u.ctx()
     c.ensure_workspace(N, g, K)
     ld = cc.cc_tensor_scores_ld(K)
@@ -186,6 +218,7 @@ def test_tensor_scores_obey_the_rounding_model(g, kind):
     cc.cc_tensor_scores(c, u.half_dev(X), N, g, u.dev(C), K, out)
     cc.cc_poll_status(c)
     got = out.cpu().numpy().astype(np.float64)[:, :K]
+    del out
     assert np.isfinite(got).all()
     Xd, Cd = X.astype(np.float64), C.astype(np.float64)
     csq = (Cd ** 2).sum(1)
@@ -203,8 +236,46 @@ def test_tensor_scores_obey_the_rounding_model(g, kind):
     absolute = inv_s * (2.0 ** -14 * np.abs(Xd).sum(1)[:, None] + norm_abs)
     err = np.abs(got - exact)
     worst = float(((err - absolute).clip(0) / rel).max())
-    print("g=%d %s: worst error %.2f units (bound %d), scale 2^%d" % (g, kind, worst, units, k))
-    assert worst <= units / 2
+    print("g=%d %s: worst error %.2f units (bound %d), scale 2^%d, %d scores" % (g, kind, worst, units, k, N * K))
+    assert worst <= units / 3
+
+
+@pytest.mark.parametrize("g,K", [(4, 1000), (8, 300), (16, 65536), (5, 64)])
+def test_finish_kernel_alone_is_right_on_good_scan_results_and_safe_on_garbage(g, K):
+    """The second kernel of the tensor-core E-step reads the winning chunk of every point from the scan's
+    output.  A scan CTA that gave up on a bounded wait writes nothing, so that word can be anything: run
+    the kernel alone on (a) the oracle's chunks -- it must find the oracle's centroid up to FP32
+    near-ties -- and (b) arbitrary bit patterns -- it must stay inside its tables and return codes < K."""
+    cc, u = _cc(), _u()
+    N = 20000
+    X = wl.make_points(N, g, 800 + g)
+    C = wl.make_codebook(K, g, 900 + g)
+    o_idx, d1, _ = oracle.assign(X, C)
+    c = u.ctx()
+    c.ensure_workspace(N, g, K)
+    Xd, Cd = u.half_dev(X), u.dev(C)
+    idx = torch.empty(N, dtype=torch.uint16, device="cuda")
+    dist = torch.empty(N, dtype=torch.float32, device="cuda")
+    scan = np.zeros((N, 2), dtype=np.float32)
+    scan[:, 0] = np.inf
+    scan[:, 1] = (o_idx // 64).astype(np.int32).view(np.float32)
+    cc.cc_tensor_finish_only(c, Xd, N, g, Cd, K, u.dev(scan), idx, dist)
+    cc.cc_poll_status(c)
+    got = u.u16_np(idx).astype(np.int32)
+    assert np.array_equal(got // 64, o_idx // 64)
+    d_got = dist.cpu().numpy().astype(np.float64)
+    assert np.all(d_got <= d1 * (1 + 1e-5) + 1e-30)                 # the chunk's best up to FP32 rounding
+    assert np.mean(got == o_idx) > 0.999
+    rng = np.random.default_rng(g)
+    junk = rng.integers(-2 ** 31, 2 ** 31, (N, 2), dtype=np.int64).astype(np.int32)
+    junk[::7, 1] = -1
+    junk[::11, 1] = 2 ** 31 - 1
+    junk[::13, 1] = (K + 63) // 64                                  # one past the last chunk
+    cc.cc_tensor_finish_only(c, Xd, N, g, Cd, K, u.dev(junk.view(np.float32)), idx, dist)
+    cc.cc_poll_status(c)                                            # no fault, no status bit
+    got = u.u16_np(idx).astype(np.int32)
+    assert got.min() >= 0 and got.max() < K
+    assert np.isfinite(dist.cpu().numpy()).all()
 
 
 def test_assign_exact_ties_and_duplicates_take_lowest_index():
@@ -473,43 +544,7 @@ def test_finalize_decode_identity_and_compress_host():
             u.centroid_rel_err(C16n.astype(np.float32), oracle.to_half(C_or).astype(np.float32), X) < 2e-3
 
 
-# ------------------------------------------------------------------ full-size workloads
-
-def test_cfg2_full_size_lockstep_then_free_run():
-    """The benchmark workload at its full size: first iteration checked on every point, the
-    following ones on a seeded sample; free-running objectives compared over 4 iterations."""
-    u = _u()
-    w = wl.WORKLOADS["cfg2_4096x4096_g4_k4096"]
-    W = wl.make_matrix(w.matrices[0])
-    X = oracle.reshape_subvectors(W, w.g)
-    N = len(X)
-    C0 = oracle.init_codebook(X, w.K, w.matrices[0].init_seed)
-    C1, trace1, tol1 = _lockstep(X, C0, 1)
-    sel = wl.subset_positions(N, 0.02, 77)
-    C3, trace3, tol3 = _lockstep(X, C1, 2, sel=sel)
-    print("cfg2 tolerated near-ties: full %d, sampled %d" % (tol1, tol3))
-    C_fit, idx_fit, dist_fit, counts_fit, trace_fit = _gpu_fit(X, C0, 4)
-    obj_or = oracle.fit(X, C0, 4)[4]
-    assert np.allclose(trace_fit, obj_or, rtol=u.REL_OBJECTIVE)
-    assert np.array_equal(trace_fit[:3], np.array(trace1 + trace3))
-
-
-@pytest.mark.parametrize("name,mat,frac", [("cfg3_4096x11008_g8_k65536", 0, 0.0008),
-                                           ("cfg5_layer7b_g16_k65536", 0, 0.002),
-                                           ("cfg5_layer7b_g16_k65536", 6, 0.0008)])
-def test_large_k_workloads_sampled(name, mat, frac):
-    """K = 65536 at full N: two iterations, the oracle checks a seeded sample of the points
-    against all centroids and runs its M-step on all points."""
-    u = _u()
-    w = wl.WORKLOADS[name]
-    spec = w.matrices[mat]
-    X = oracle.reshape_subvectors(wl.make_matrix(spec), w.g)
-    C0 = oracle.init_codebook(X, w.K, spec.init_seed)
-    sel = wl.subset_positions(len(X), frac, 5)
-    C, trace, tol = _lockstep(X, C0, 2, sel=sel)
-    print(name, spec.name, "tolerated near-ties on the sample:", tol, "objective", trace)
-    assert trace[1] < trace[0]
-
+# ------------------------------------------------------------------ the paper's own (g, n) settings
 
 @pytest.mark.parametrize("name,frac", [("grid_g6_n65500", 0.001), ("grid_g9_n65500", 0.001),
                                        ("grid_g5_n50000", 0.001), ("grid_g7_n35000", 0.001)])
@@ -550,17 +585,6 @@ def test_paper_grid_settings_padded_and_sampled(name, frac):
     assert pad > 0 and pad_share > 0
     assert tr[-1].item() == pytest.approx(err + pad_share, rel=1e-7)   # dist is rounded to FP32 per point
     u.check_assign_against_oracle(X, C16n.astype(np.float32), idxn, None, sel)
-
-
-def test_cfg4_full_size_one_iteration_sampled():
-    u = _u()
-    w = wl.WORKLOADS["cfg4_8192x28672_g4_k65536"]
-    spec = w.matrices[0]
-    X = oracle.reshape_subvectors(wl.make_matrix(spec), w.g)
-    C0 = oracle.init_codebook(X, w.K, spec.init_seed)
-    sel = wl.subset_positions(len(X), 0.0002, 5)
-    C, trace, tol = _lockstep(X, C0, 1, sel=sel)
-    print("cfg4 tolerated near-ties on the sample:", tol, "objective", trace)
 
 
 # ------------------------------------------------------------------ bounded device-side waits

@@ -15,6 +15,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_2503_13089_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -51,6 +52,9 @@ def test_update_static_matches_update_on_two_calls_in_a_row():
         assert np.array_equal(counts_st, counts_ref)
         assert u.centroid_rel_err(C_st, C_ref, X) <= u.REL_CENTROID
         assert np.array_equal(C_st.view(np.uint32), C_ref.view(np.uint32))
+        C_or, counts_or = oracle.update(X, idx, C_prev)              # and the CPU oracle says the same
+        assert np.array_equal(counts_st.astype(np.int64), counts_or.astype(np.int64))
+        assert np.array_equal(C_st.view(np.uint32), C_or.view(np.uint32))
         empty = counts_ref == 0
         assert empty.any() and np.array_equal(C_st[empty].view(np.uint32), C_prev[empty].view(np.uint32))
 
@@ -73,3 +77,36 @@ def test_update_static_rejects_sizes_beyond_its_fixed_capacity():
     cc.cc_update_static(0, X, 16, g, idx, K, C[:K], counts[:K])
     torch.cuda.synchronize()
     assert int(counts[0].item()) == 16 and int(counts[1:K].sum().item()) == 0
+
+
+def test_update_static_at_full_capacity_and_without_touching_the_allocator():
+    """K * g exactly at the fixed capacity with members in the very last cluster (the last words of
+    the array are used), compared with the oracle; and a warm call must leave the device's free
+    memory as it found it -- the point of the entry point is that it never allocates."""
+    from paper_2503_13089_b200 import binding as cc
+    from tests import gpu_util as u
+    g = 4
+    K = cc.UPDATE_STATIC_MAX_KG // g
+    rng = np.random.default_rng(9)
+    X = wl.make_points(50000, g, 35)
+    idx = rng.integers(0, K, len(X)).astype(np.int32)
+    idx[-3:] = K - 1
+    C_prev = wl.make_codebook(K, g, 36)
+    Xd = u.half_dev(X)
+    idxd = torch.from_numpy(idx.astype(np.uint16).view(np.int16)).cuda().view(torch.uint16)
+    Cd = u.dev(C_prev)
+    counts = torch.empty(K, dtype=torch.int32, device="cuda")
+    cc.cc_update_static(0, Xd, len(X), g, idxd, K, Cd, counts)       # first call on the device: set-up
+    torch.cuda.synchronize()
+    C_or, counts_or = oracle.update(X, idx, C_prev)
+    assert counts_or[K - 1] >= 3
+    assert np.array_equal(counts.cpu().numpy().astype(np.int64), counts_or.astype(np.int64))
+    assert np.array_equal(Cd.cpu().numpy().view(np.uint32), C_or.view(np.uint32))
+    Cd.copy_(torch.from_numpy(C_prev))
+    torch.cuda.synchronize()
+    free_before, _ = torch.cuda.mem_get_info()
+    cc.cc_update_static(0, Xd, len(X), g, idxd, K, Cd, counts)       # warm call
+    torch.cuda.synchronize()
+    free_after, _ = torch.cuda.mem_get_info()
+    assert free_after == free_before
+    assert np.array_equal(Cd.cpu().numpy().view(np.uint32), C_or.view(np.uint32))

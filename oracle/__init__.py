@@ -51,6 +51,9 @@ def _load():
         lib.oc_update.argtypes = [vp, i64, i32, vp, i32, vp, vp]
         lib.oc_codebook_grad.argtypes = [vp, i64, i32, vp, i32, vp]
         lib.oc_fit.argtypes = [vp, i64, i32, i32, i32, vp, vp, vp, vp, vp]
+        lib.oc_linear_forward.argtypes = [vp, i64, vp, i32, vp, i64, i64, vp, vp]
+        lib.oc_quantize_codebook.argtypes = [vp, i64, i32, vp, vp, vp]
+        lib.oc_split_empty.argtypes = [vp, i32, i32, vp]
         lib.oc_float_to_half.argtypes = [vp, i64, vp]
         lib.oc_half_to_double.argtypes = [vp, i64, vp]
         _lib = lib
@@ -199,3 +202,94 @@ def finalize(X: np.ndarray, C: np.ndarray):
     C16 = to_half(C)
     idx, d1, _ = assign(X, C16.astype(np.float32))
     return C16, idx, d1, float(np.sum(d1))
+
+
+def linear_forward(x: np.ndarray, C16: np.ndarray, idx: np.ndarray, d_out: int, d_in: int,
+                   bias: Optional[np.ndarray] = None) -> np.ndarray:
+    """Forward of the compressed linear layer: y = x . codebook[code].view(in, -1)[:, :d_out] (+ bias).
+
+    x: M x d_in FP16.  Returns M x d_out float64."""
+    x = _half(x)
+    C16 = _half(C16)
+    M = x.shape[0]
+    K, g = C16.shape
+    assert x.shape[1] == d_in
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    assert idx.size == num_subvectors(d_out, d_in, g) and idx.min() >= 0 and idx.max() < K
+    if bias is not None:
+        bias = np.ascontiguousarray(bias, dtype=np.float32)
+        assert bias.shape == (d_out,)
+    y = np.empty((M, d_out), dtype=np.float64)
+    _load().oc_linear_forward(_p(x), M, _p(C16), g, _p(idx), d_out, d_in, _p(bias), _p(y))
+    return y
+
+
+def quantize_codebook(C16: np.ndarray, bits: int):
+    """Uniform symmetric quantisation of the stored codebook to `bits` (8 or 4) bits.
+
+    Returns (q int8 of C16's shape, scale float32, dequantised FP16 codebook)."""
+    C16 = _half(C16)
+    assert bits in (8, 4)
+    q = np.empty(C16.shape, dtype=np.int8)
+    scale = np.empty(1, dtype=np.float32)
+    deq = np.empty(C16.shape, dtype=np.float16)
+    _load().oc_quantize_codebook(_p(C16), C16.size, bits, _p(q), _p(scale), _p(deq))
+    return q, float(scale[0]), deq
+
+
+def pack_nibbles(q: np.ndarray) -> np.ndarray:
+    """Storage format of a 4-bit codebook: element 2k in the low nibble of byte k, element 2k+1 in the
+    high nibble (two's complement nibbles); an odd element count leaves the last high nibble 0."""
+    flat = q.reshape(-1).astype(np.int16) & 0xF
+    if flat.size % 2:
+        flat = np.concatenate([flat, np.zeros(1, np.int16)])
+    return (flat[0::2] | (flat[1::2] << 4)).astype(np.uint8)
+
+
+def split_empty(C: np.ndarray, counts: np.ndarray) -> np.ndarray:
+    """Second empty-cluster rule applied to the centroids of one M-step; returns the new centroids."""
+    C = np.array(C, dtype=np.float32, order="C", copy=True)
+    counts = np.ascontiguousarray(counts, dtype=np.int64)
+    K, g = C.shape
+    assert counts.shape == (K,)
+    _load().oc_split_empty(_p(C), K, g, _p(counts))
+    return C
+
+
+EMPTY_KEEP, EMPTY_SPLIT = 0, 1
+
+
+def fit_ex(X: np.ndarray, C0: np.ndarray, iters: int, empty_rule: int = EMPTY_KEEP):
+    """Lloyd loop with a choice of empty-cluster rule, written with the one-step primitives.
+
+    Returns (C, idx of the last E-step, d1, counts, objective[iters])."""
+    C = np.array(C0, dtype=np.float32, order="C", copy=True)
+    obj = np.empty(iters, dtype=np.float64)
+    idx = d1 = counts = None
+    for it in range(iters):
+        idx, d1, _ = assign(X, C)
+        obj[it] = float(np.sum(d1))
+        C, counts = update(X, idx, C)
+        if empty_rule == EMPTY_SPLIT:
+            C = split_empty(C, counts)
+    return C, idx, d1, counts, obj
+
+
+def train_positions(N: int, K: int, max_points_per_centroid: int, seed: int) -> Optional[np.ndarray]:
+    """Training-set subsampling: when N exceeds max_points_per_centroid * K, the Lloyd loop runs on
+    that many points, drawn as distinct positions by the same seeded partial shuffle that draws the
+    initial centroids; None when all points are used."""
+    n = max_points_per_centroid * K
+    if n >= N:
+        return None
+    return init_positions(N, n, seed)
+
+
+def fit_sampled(X: np.ndarray, C0: np.ndarray, iters: int, max_points_per_centroid: int, seed: int):
+    """Lloyd loop on the subsampled training set, then one E-step over ALL points against the fitted
+    codebook.  Returns (C, idx over all points, d1 over all points, training counts, objective[iters])."""
+    pos = train_positions(len(X), C0.shape[0], max_points_per_centroid, seed)
+    Xt = X if pos is None else np.ascontiguousarray(X[pos])
+    C, _, _, counts, obj = fit(Xt, C0, iters)
+    idx, d1, _ = assign(X, C)
+    return C, idx, d1, counts, obj

@@ -242,3 +242,78 @@ void oc_fit(const uint16_t* X, int64_t N, int g, int K, int iters, float* C, int
         oc_update(X, N, g, idx, K, C, counts);
     }
 }
+
+/* ---- Forward of the compressed linear layer (appendix listing) -------------------
+ * weight = codebook[code] viewed as (in_features, out_features + pad) with the padded columns
+ * dropped; out = x . weight (+ bias).  x: M x d_in FP16 (row-major), y: M x d_out doubles,
+ * y[m][o] = sum_i x[m][i] * weight[i][o] + bias[o], summed over i in increasing order.     */
+void oc_linear_forward(const uint16_t* x, int64_t M, const uint16_t* C16, int g, const int32_t* idx,
+                       int64_t d_out, int64_t d_in, const float* bias, double* y) {
+    int64_t out_pad = padded(d_out, g);
+    for (int64_t m = 0; m < M; ++m)
+        for (int64_t o = 0; o < d_out; ++o) {
+            double s = 0.0;
+            for (int64_t i = 0; i < d_in; ++i) {
+                int64_t flat = i * out_pad + o;            /* position in the (in, out_pad) view */
+                double w = half_to_double(C16[(int64_t)idx[flat / g] * g + flat % g]);
+                s += half_to_double(x[m * d_in + i]) * w;
+            }
+            y[m * d_out + o] = bias ? s + (double)bias[o] : s;
+        }
+}
+
+/* ---- Uniform quantisation of the codebook (Section 5.3 "Inference latency": the FP16 codebook
+ * may be quantised uniformly to 8 or 4 bits; the grid is the symmetric uniform one of the related-
+ * work section: q = clamp(round-to-nearest(c / s), -2^(b-1), 2^(b-1) - 1)).  One scale for the whole
+ * codebook.  Reading of the scale: s = max|c| / (2^(b-1) - 1), so that the grid spans the values (the
+ * printed denominator 2^b - 1 would clip every value above half of the range).  The paper fixes no
+ * precision; taken here: s and c / s in float (IEEE single, round-to-nearest), rounding of the
+ * quotient to the nearest integer with ties to even.  deq = FP16(q * s) (float product, RNE).    */
+void oc_quantize_codebook(const uint16_t* C16, int64_t n, int bits, int8_t* q, float* scale, uint16_t* deq) {
+    float maxabs = 0.0f;
+    for (int64_t e = 0; e < n; ++e) {
+        float a = (float)fabs(half_to_double(C16[e]));
+        if (a > maxabs) maxabs = a;
+    }
+    int L = (1 << (bits - 1)) - 1;
+    float s = maxabs > 0.0f ? maxabs / (float)L : 1.0f;
+    *scale = s;
+    for (int64_t e = 0; e < n; ++e) {
+        float c = (float)half_to_double(C16[e]);
+        float t = c / s;
+        double r = nearbyint((double)t);                   /* default rounding mode: ties to even */
+        if (r < -(double)(L + 1)) r = -(double)(L + 1);
+        if (r > (double)L) r = (double)L;
+        q[e] = (int8_t)r;
+        if (deq) deq[e] = float_to_half_rne((float)q[e] * s);
+    }
+}
+
+/* ---- Second empty-cluster rule: split the most populated cluster ---------------------
+ * The paper does not say what happens to a cluster that loses all its points; the default rule of
+ * this oracle keeps its centroid.  This optional rule re-seeds it instead, the way k-means
+ * libraries commonly do.  After the means: for every empty cluster e in increasing order, the donor
+ * d is the cluster with the largest working count (lowest index among equals); if that count is
+ * below 2, e keeps its centroid.  Otherwise c_e = c_d, then coordinate t of c_e is multiplied by
+ * (1 + eps) and that of c_d by (1 - eps) for even t, the other way round for odd t (eps = 2^-10,
+ * float products), and the working counts become n_e = floor(n_d / 2), n_d = n_d - n_e.
+ * `counts` (true member counts) is not changed.                                               */
+void oc_split_empty(float* C, int K, int g, const int64_t* counts) {
+    int64_t* work = (int64_t*)malloc(sizeof(int64_t) * (size_t)K);
+    memcpy(work, counts, sizeof(int64_t) * (size_t)K);
+    const float up = 1.0f + 0.0009765625f, down = 1.0f - 0.0009765625f;
+    for (int e = 0; e < K; ++e) {
+        if (counts[e] != 0) continue;
+        int d = 0;
+        for (int j = 1; j < K; ++j) if (work[j] > work[d]) d = j;
+        if (work[d] < 2) continue;
+        for (int t = 0; t < g; ++t) {
+            float c = C[(int64_t)d * g + t];
+            C[(int64_t)e * g + t] = c * ((t & 1) ? down : up);
+            C[(int64_t)d * g + t] = c * ((t & 1) ? up : down);
+        }
+        work[e] = work[d] / 2;
+        work[d] -= work[e];
+    }
+    free(work);
+}

@@ -409,3 +409,145 @@ def test_codebook_grad_against_exact_rationals_autograd_and_the_m_step():
     # K = 1: the column sums
     assert np.array_equal(oracle.codebook_grad(a, np.zeros(N, np.int32), 1)[0],
                           a.astype(np.float64).sum(0).astype(np.float32))
+
+
+# ---------------------------------------------------------------- compressed linear layer (appendix listing)
+
+def _layer_case(M, d_out, d_in, g, K, seed):
+    rng = np.random.default_rng(seed)
+    x = rng.standard_normal((M, d_in)).astype(np.float16)
+    C16 = (rng.standard_normal((K, g)) * 0.1).astype(np.float16)
+    idx = rng.integers(0, K, oracle.num_subvectors(d_out, d_in, g)).astype(np.int32)
+    return x, C16, idx
+
+
+@pytest.mark.parametrize("M,d_out,d_in,g,K", [(3, 8, 5, 4, 7), (2, 10, 7, 4, 9), (5, 9, 16, 6, 33), (1, 64, 48, 16, 5),
+                                               (4, 7, 3, 9, 4)])
+def test_linear_forward_is_the_listing(M, d_out, d_in, g, K):
+    """codebook[code].view(in_features, -1) with the padded columns dropped, then x @ weight + bias:
+    written here with numpy indexing and a library matmul in float64."""
+    x, C16, idx = _layer_case(M, d_out, d_in, g, K, M + d_out + d_in)
+    bias = np.random.default_rng(1).standard_normal(d_out).astype(np.float32)
+    weight = C16[idx].reshape(d_in, -1)[:, :d_out].astype(np.float64)
+    want = x.astype(np.float64) @ weight
+    assert np.allclose(oracle.linear_forward(x, C16, idx, d_out, d_in), want, rtol=1e-13, atol=1e-13)
+    assert np.allclose(oracle.linear_forward(x, C16, idx, d_out, d_in, bias), want + bias.astype(np.float64),
+                       rtol=1e-13, atol=1e-13)
+    # the same weight is what decode lays out as a (d_out, d_in) matrix
+    W_hat = oracle.decode(C16, idx, d_out, d_in).astype(np.float64)
+    assert np.allclose(oracle.linear_forward(x, C16, idx, d_out, d_in), x.astype(np.float64) @ W_hat.T,
+                       rtol=1e-13, atol=1e-13)
+
+
+def test_linear_forward_exact_rationals_and_unit_inputs():
+    x, C16, idx = _layer_case(2, 6, 5, 4, 5, 3)
+    d_out, d_in, g = 6, 5, 4
+    got = oracle.linear_forward(x, C16, idx, d_out, d_in)
+    out_pad = 8
+    for m in range(2):
+        for o in range(d_out):
+            s = Fraction(0)
+            for i in range(d_in):
+                flat = i * out_pad + o
+                s += Fraction(float(x[m, i])) * Fraction(float(C16[idx[flat // g], flat % g]))
+            assert got[m, o] == pytest.approx(float(s), rel=1e-14, abs=1e-300)
+    # unit vectors as inputs read the weight's rows: row i of the (in, out) weight = column i of decode
+    eye = np.eye(d_in, dtype=np.float16)
+    assert np.array_equal(oracle.linear_forward(eye, C16, idx, d_out, d_in),
+                          oracle.decode(C16, idx, d_out, d_in).astype(np.float64).T)
+    # zero input leaves the bias
+    b = np.arange(d_out, dtype=np.float32)
+    assert np.array_equal(oracle.linear_forward(np.zeros((1, d_in), np.float16), C16, idx, d_out, d_in, b)[0], b)
+
+
+# ---------------------------------------------------------------- uniform codebook quantisation (Section 5.3)
+
+@pytest.mark.parametrize("bits", [8, 4])
+def test_quantize_codebook_grid_range_and_error_bound(bits):
+    rng = np.random.default_rng(bits)
+    C16 = (rng.standard_t(3.0, (500, 6)) * 0.02).astype(np.float16)
+    q, s, deq = oracle.quantize_codebook(C16, bits)
+    L = 2 ** (bits - 1) - 1
+    c = C16.astype(np.float64)
+    assert s == np.float32(np.float32(np.abs(c).max()) / np.float32(L))
+    assert q.max() == L or q.min() == -L                       # the largest magnitude sits on the last level
+    assert q.min() >= -L and q.max() <= L                      # -2^(b-1) is never needed on a symmetric grid
+    assert np.all(np.abs(c - q.astype(np.float64) * s) <= 0.5 * s * (1 + 1e-6))   # round to NEAREST
+    assert len(np.unique(q)) <= 2 ** bits
+    q2, s2, _ = oracle.quantize_codebook((-C16).astype(np.float16), bits)
+    assert s2 == s and np.array_equal(q2, -q)                  # symmetric grid, ties to even
+    assert np.allclose(deq.astype(np.float64), q * np.float64(s), rtol=2.0 ** -11, atol=2.0 ** -25)
+
+
+def test_quantize_codebook_worked_examples():
+    # values that already sit on a power-of-two grid come back as themselves
+    C16 = np.array([[-1.75, 0.0, 0.25, 1.5], [1.75, -0.5, 0.75, -1.25]], dtype=np.float16)   # max 1.75 = 7 * 0.25
+    q, s, deq = oracle.quantize_codebook(C16, 4)
+    assert s == 0.25 and np.array_equal(q, (C16.astype(np.float64) / 0.25).astype(np.int8))
+    assert np.array_equal(deq, C16)
+    # exact halves round to the even level: with s = 1/4, 0.125 -> 0.5 -> 0, 0.375 -> 1.5 -> 2, 0.625 -> 2.5 -> 2
+    C16 = np.array([[1.75, 0.125, 0.375, 0.625, -0.125, -0.375]], dtype=np.float16)
+    q, s, _ = oracle.quantize_codebook(C16, 4)
+    assert s == 0.25 and q.tolist() == [[7, 0, 2, 2, 0, -2]]
+    # 8 bits: 127 levels each side
+    C16 = np.array([[127.0, -64.0, 0.5, 1.5, 2.5, -126.6]], dtype=np.float16)
+    q, s, _ = oracle.quantize_codebook(C16, 8)
+    assert s == 1.0 and q.tolist() == [[127, -64, 0, 2, 2, -127]]      # FP16(-126.6) = -126.625
+    # an all-zero codebook
+    q, s, deq = oracle.quantize_codebook(np.zeros((3, 4), np.float16), 8)
+    assert s == 1.0 and not q.any() and not deq.any()
+    # nibble packing: low nibble first, two's complement
+    assert oracle.pack_nibbles(np.array([7, -7, 0, -1, 3], np.int8)).tolist() == [0x97, 0xF0, 0x03]
+
+
+# ---------------------------------------------------------------- second empty-cluster rule
+
+def test_split_empty_worked_example():
+    """K = 4, g = 2, counts (5, 0, 3, 0): cluster 1 takes half of cluster 0; then the working counts are
+    (3, 2, 3, 0), clusters 0 and 2 tie and the lower index donates again.  Centroid 0 = (1024, 2048) so
+    that every product with 1 +- 2^-10 is exact."""
+    C = np.array([[1024.0, 2048.0], [5.0, 5.0], [-3.0, 7.0], [9.0, 9.0]], dtype=np.float32)
+    out = oracle.split_empty(C, np.array([5, 0, 3, 0]))
+    assert out[1].tolist() == [1025.0, 2046.0]
+    assert out[3].tolist() == [1023.0 + 1023.0 / 1024.0, 2050.0 - 2050.0 / 1024.0]
+    assert out[0].tolist() == [1023.0 - 1023.0 / 1024.0, 2050.0 + 2050.0 / 1024.0]
+    assert out[2].tolist() == [-3.0, 7.0]
+    # nobody can donate: every cluster has at most one point
+    C2 = np.arange(8, dtype=np.float32).reshape(4, 2)
+    assert np.array_equal(oracle.split_empty(C2, np.array([1, 0, 1, 0])), C2)
+    # no empty cluster: nothing moves
+    assert np.array_equal(oracle.split_empty(C2, np.array([4, 2, 1, 9])), C2)
+
+
+def test_split_rule_fills_empty_clusters_and_lowers_the_objective():
+    X, labels, centres = wl.make_blobs(6, 200, 4, seed=4, sep=1.0, sigma=0.02)
+    first = np.array([np.flatnonzero(labels == b)[0] for b in range(6)])
+    C0 = X[first].astype(np.float32)
+    C0[5] = 50.0                                        # one start far from every point: its cluster stays empty
+    C_keep, idx_k, _, counts_k, obj_k = oracle.fit_ex(X, C0, 6, oracle.EMPTY_KEEP)
+    C_ref, idx_r, _, counts_r, obj_r = oracle.fit(X, C0, 6)
+    assert np.array_equal(C_keep, C_ref) and np.allclose(obj_k, obj_r, rtol=1e-13)   # rule 0 is the plain loop
+    assert counts_k[5] == 0 and np.array_equal(C_keep[5], C0[5])
+    C_split, idx_s, _, counts_s, obj_s = oracle.fit_ex(X, C0, 6, oracle.EMPTY_SPLIT)
+    assert counts_s.min() > 0 and counts_s.sum() == len(X)
+    assert obj_s[-1] < obj_k[-1]
+
+
+# ---------------------------------------------------------------- training-set subsampling
+
+def test_fit_sampled_reduces_to_the_plain_loop_and_uses_the_drawn_rows():
+    X = wl.make_points(3000, 4, 21)
+    C0 = oracle.init_codebook(X, 10, 3)
+    # enough room for every point: the plain loop followed by one E-step
+    C, idx, d1, counts, obj = oracle.fit_sampled(X, C0, 3, 300, 9)
+    C_ref, _, _, counts_ref, obj_ref = oracle.fit(X, C0, 3)
+    assert np.array_equal(C, C_ref) and np.array_equal(obj, obj_ref) and np.array_equal(counts, counts_ref)
+    assert np.array_equal(idx, oracle.assign(X, C_ref)[0])
+    # 50 points per centroid: 500 distinct seeded positions are the training set
+    pos = oracle.train_positions(3000, 10, 50, 9)
+    assert len(pos) == 500 and len(set(pos.tolist())) == 500 and np.array_equal(pos, oracle.init_positions(3000, 500, 9))
+    C, idx, d1, counts, obj = oracle.fit_sampled(X, C0, 3, 50, 9)
+    C_t, _, _, counts_t, obj_t = oracle.fit(np.ascontiguousarray(X[pos]), C0, 3)
+    assert np.array_equal(C, C_t) and counts.sum() == 500 and np.array_equal(obj, obj_t)
+    assert len(idx) == 3000 and np.array_equal(idx, oracle.assign(X, C)[0])
+    assert oracle.train_positions(3000, 10, 300, 9) is None

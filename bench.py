@@ -369,7 +369,8 @@ def run_kernel_mode(a):
     from paper_2503_13089_b200 import binding as cc
     N, g, K = a.N, a.g, a.K
     ctx = cc.Context(0)
-    ctx.ensure_workspace(N, g, K)
+    d_out, d_in = g * 1024, N // 1024
+    ctx.ensure_workspace(N, g, K, at_least=cc.cc_linear_workspace_bytes(ctx, a.M, d_out, max(d_in, 1)) if a.kernel == "linear" else 0)
     cc.cc_set_path(ctx, {"auto": 0, "ffma": 1, "tensor": 2}[a.path])
     Xn = wl.make_points(N, g, 1)
     X = torch.from_numpy(Xn.view(np.int16)).cuda().view(torch.float16)
@@ -381,7 +382,6 @@ def run_kernel_mode(a):
     obj = torch.zeros(1, dtype=torch.float64, device="cuda")
     nres = torch.zeros(1, dtype=torch.int64, device="cuda")
     C16 = torch.empty((K, g), dtype=torch.float16, device="cuda")
-    d_out, d_in = g * 1024, N // 1024
     if a.kernel in ("decode", "reshape", "linear"):
         assert d_in * 1024 == N, "N must be a multiple of 1024 for the reshape / decode / linear cases"
     W = torch.empty((d_out, d_in), dtype=torch.float16, device="cuda")
@@ -489,8 +489,12 @@ def main():
     else:
         ceiling_for = lambda g: ceiling_scores                      # noqa: E731
 
-    # ---------------- headline workload: rank r clusters the workload's matrices with seeds shifted by r
-    specs = sharding.matrices_for_rank(w, rank)
+    # ---------------- headline workload.  The job is `world` copies of the workload's matrices (copy r with
+    # seeds shifted by r: weak scaling); the library's size-balanced scheduler says which of them this rank
+    # clusters.  Nothing is exchanged between ranks.
+    job = [m for r in range(world) for m in sharding.matrices_for_rank(w, r)]
+    mine = cc.cc_schedule_matrices([w.n_subvectors(m) for m in job], world, rank)
+    specs = tuple(job[i] for i in mine)
     run = Runner(cc, torch, ctx, w, specs, layout)
     for _ in range(args.warmup):
         flush.zero_()

@@ -101,7 +101,8 @@ int64_t cc_launch_count(const cc_ctx* ctx);
 #define CC_KERNEL_OTHER 8
 #define CC_KERNEL_ASSIGN_FINISH 9 /* tensor path: index, distance, near-tie flag per point */
 #define CC_KERNEL_UPDATE_DELTA 10  /* M-step inside cc_fit: only the points whose code changed */
-#define CC_KERNEL_CLASSES 11
+#define CC_KERNEL_LINEAR 11        /* forward of the compressed linear layer (GEMM + split reduction) */
+#define CC_KERNEL_CLASSES 12
 cc_status cc_profile_enable(cc_ctx* ctx, int on);
 cc_status cc_profile_read(cc_ctx* ctx, double* total_ms_host, int64_t* launches_host);
 
@@ -262,6 +263,60 @@ cc_status cc_codebook_grad(cc_ctx* ctx, const uint16_t* dX, int64_t N, int g, co
 cc_status cc_fit(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, int K, int iters, float* C,
                  uint16_t* idx, float* dist, int32_t* counts, double* objective_trace, void* stream);
 
+/* What the M-step does with a cluster that has no member (the paper does not say; it runs its
+ * k-means library with default settings).  CC_EMPTY_KEEP (default): the centroid is kept bit for bit.
+ * CC_EMPTY_SPLIT_LARGEST: after the means, every empty cluster e, in increasing order, is re-seeded from
+ * the most populated cluster d (largest working count, lowest index among equals; nothing happens once
+ * that count is below 2): c_e = c_d, then coordinate t of c_e is multiplied by 1 + 2^-10 and that of c_d
+ * by 1 - 2^-10 for even t and the other way round for odd t (FP32 products), and the working counts become
+ * n_e = floor(n_d / 2), n_d = n_d - n_e.  `counts` always reports the true member counts.  Applies to
+ * cc_update, cc_fit, cc_fit_sampled and cc_compress_host on this context (not to cc_update_static). */
+#define CC_EMPTY_KEEP 0
+#define CC_EMPTY_SPLIT_LARGEST 1
+cc_status cc_set_empty_rule(cc_ctx* ctx, int rule);
+
+/* Lloyd loop on a subsample of the points, then one E-step over all of them (k-means libraries, the
+ * paper's included, by default train on at most a fixed number of points per centroid; the paper
+ * states no such number, so it is an argument here).  n = cc_train_points(N, K, max_points_per_centroid)
+ * = min(N, max_points_per_centroid * K) distinct positions are drawn by the seeded partial shuffle of
+ * cc_init_positions (the first n entries for `seed`), those rows are copied in that order to X_train
+ * (device scratch of n x g FP16, 16-byte aligned; may be NULL when n == N), cc_fit runs on them, and a
+ * final cc_assign over all N points against the fitted codebook fills idx / dist (N entries each; dist
+ * may be NULL).  counts and objective_trace are those of the training set.  C: in = initial codebook. */
+int64_t cc_train_points(int64_t N, int K, int max_points_per_centroid);
+cc_status cc_fit_sampled(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, int K, int iters, int max_points_per_centroid,
+                         uint64_t seed, uint16_t* X_train, float* C, uint16_t* idx, float* dist, int32_t* counts,
+                         double* objective_trace, void* stream);
+
+/* Uniform quantisation of the stored codebook (Section 5.3 "Inference latency": for inference the FP16
+ * codebook may be quantised uniformly to 8 or 4 bits) on the symmetric uniform grid of the related-work
+ * section: q = clamp(round-to-nearest(c / s), -2^(b-1), 2^(b-1) - 1), one scale s for the whole codebook.
+ * Reading of the scale: s = max|c| / (2^(b-1) - 1), so that the grid spans the values (the printed
+ * denominator 2^b - 1 would clip everything above half of the range); s = 1 for an all-zero codebook.
+ * s and c / s are IEEE single precision, the quotient is rounded to the nearest integer, ties to even.
+ * bits: 8 or 4.  q (out): K * g signed bytes (8 bits), or ceil(K * g / 2) bytes holding element 2k in
+ * the low and element 2k + 1 in the high nibble, two's complement (4 bits).  scale (out, device): one
+ * float.  C16_dequantized (out, may be NULL): K x g FP16 = round-to-nearest-even of q * s, usable with
+ * cc_decode and cc_linear_forward.  Needs a workspace of at least 256 bytes. */
+cc_status cc_quantize_codebook(cc_ctx* ctx, const uint16_t* C16, int K, int g, int bits, uint8_t* q, float* scale,
+                               uint16_t* C16_dequantized, void* stream);
+
+/* The clustering of different weight matrices is independent (remark at the end of Section 3.1), so a
+ * model is spread over GPUs matrix by matrix with nothing exchanged.  cc_schedule_matrices (host only):
+ * longest-processing-time-first split of n matrices with costs sizes_host[i] (e.g. their numbers of
+ * sub-vectors) over `world` ranks -- matrices by decreasing cost, lower index first among equals, each to
+ * the rank with the smallest load so far, lowest rank among equals; writes the indices that fall to
+ * `rank`, in increasing order, to mine_host (room for n) and their number to *n_mine_host.
+ * cc_compress_many runs cc_compress_host on each of n matrices in turn (arrays of n host pointers and
+ * sizes; objective_trace_hosts and W_hat_hosts, or single entries of them, may be NULL) and stops at
+ * the first status other than CC_OK. */
+cc_status cc_schedule_matrices(int n, const int64_t* sizes_host, int world, int rank, int32_t* mine_host,
+                               int32_t* n_mine_host);
+cc_status cc_compress_many(cc_ctx* ctx, int n, const uint16_t* const* W_hosts, const int64_t* d_outs, const int64_t* d_ins,
+                           int g, int K, int iters, const uint64_t* seeds, int layout, uint16_t* const* C16_hosts,
+                           uint16_t* const* idx_hosts, double* const* objective_trace_hosts, uint16_t* const* W_hat_hosts,
+                           void* stream);
+
 /* Section 3.1 (codes = nearest centroid of the final codebook) and Section 3.2 (FP16 storage):
  * C16 = round-to-nearest-even FP16 of C; idx / dist / objective = E-step against C16, so the
  * stored pair (C16, idx) is consistent and ||W - decode||^2 equals *objective (no padding). */
@@ -273,6 +328,22 @@ cc_status cc_finalize(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const fl
  * idx: cc_num_subvectors(...) codes, each < K. */
 cc_status cc_decode(cc_ctx* ctx, const uint16_t* C16, int K, int g, const uint16_t* idx,
                     int64_t d_out, int64_t d_in, int layout, uint16_t* W_hat, void* stream);
+
+/* Forward of the compressed linear layer, appendix listing (ClusCompLinear.forward):
+ *   weight = codebook[code].view(in_features, -1) with the padded columns dropped;  y = x . weight (+ bias).
+ * The decoded weight is never written to memory: codebook rows are gathered straight into the
+ * shared-memory operand of a tensor-core GEMM (FP16 inputs, FP32 accumulation).
+ * x: M x d_in FP16 row-major (M tokens).  C16: K x g FP16.  idx: cc_num_subvectors(d_out, d_in, g,
+ * CC_LAYOUT_PAPER_T) codes, each < K.  bias (may be NULL): d_out FP32.  y (out): M x d_out FP32
+ * row-major.  The listing keeps every tensor in a 16-bit type; here the accumulator is handed out
+ * unrounded.  Scratch: cc_linear_workspace_bytes(M, d_out, d_in) bytes of the context's workspace
+ * (cc_set_workspace; used when the in_features are split across thread blocks, which happens for
+ * small M; the partial sums are added in a fixed order, so the result is the same on every call).
+ * 1 <= M < 2^31 / d_out; x, C16, y 16-byte aligned. */
+size_t cc_linear_workspace_bytes(cc_ctx* ctx, int64_t M, int64_t d_out, int64_t d_in);
+cc_status cc_linear_forward(cc_ctx* ctx, const uint16_t* x, int64_t M, const uint16_t* C16, int K, int g,
+                            const uint16_t* idx, int64_t d_out, int64_t d_in, const float* bias, float* y,
+                            void* stream);
 
 /* Waits for `stream`, reads the device status word and clears it.  Returns CC_OK,
  * CC_ERR_NONFINITE, CC_ERR_DEVICE_TIMEOUT or CC_ERR_CUDA. */

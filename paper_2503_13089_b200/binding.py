@@ -19,6 +19,7 @@ CC_OK = 0
 LAYOUT_PAPER_T = 0
 LAYOUT_ROWS = 1
 PATH_AUTO, PATH_FFMA, PATH_TENSOR = 0, 1, 2
+EMPTY_KEEP, EMPTY_SPLIT_LARGEST = 0, 1
 
 STATUS_NAMES = {
     0: "CC_OK", 1: "CC_ERR_NULL", 2: "CC_ERR_SHAPE", 3: "CC_ERR_UNSUPPORTED_G", 4: "CC_ERR_K_RANGE",
@@ -57,8 +58,16 @@ SIGNATURES = {
     "cc_update_static": (_i32, [_i32, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp]),
     "cc_codebook_grad": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp]),
     "cc_fit": (_i32, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "cc_set_empty_rule": (_i32, [_vp, _i32]),
+    "cc_train_points": (_i64, [_i64, _i32, _i32]),
+    "cc_fit_sampled": (_i32, [_vp, _vp, _i64, _i32, _i32, _i32, _i32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
+    "cc_quantize_codebook": (_i32, [_vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp]),
+    "cc_schedule_matrices": (_i32, [_i32, _vp, _i32, _i32, _vp, _vp]),
+    "cc_compress_many": (_i32, [_vp, _i32, _vp, _vp, _vp, _i32, _i32, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp]),
     "cc_finalize": (_i32, [_vp, _vp, _i64, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _vp]),
     "cc_decode": (_i32, [_vp, _vp, _i32, _i32, _vp, _i64, _i64, _i32, _vp, _vp]),
+    "cc_linear_workspace_bytes": (_sz, [_vp, _i64, _i64, _i64]),
+    "cc_linear_forward": (_i32, [_vp, _vp, _i64, _vp, _i32, _i32, _vp, _i64, _i64, _vp, _vp, _vp]),
     "cc_poll_status": (_i32, [_vp, _vp]),
     "cc_compress_host": (_i32, [_vp, _vp, _i64, _i64, _i32, _i32, _i32, _u64, _i32, _vp, _vp, _vp, _vp, _vp]),
 }
@@ -129,8 +138,8 @@ class Context:
         except Exception:
             pass
 
-    def ensure_workspace(self, N: int, g: int, K: int) -> None:
-        need = cc_workspace_bytes(N, g, K)
+    def ensure_workspace(self, N: int, g: int, K: int, at_least: int = 0) -> None:
+        need = max(cc_workspace_bytes(N, g, K), at_least)
         if need == 0:
             raise CCError(2, "cc_workspace_bytes")
         if self._ws is None or self._ws.numel() < need:
@@ -159,7 +168,7 @@ def cc_launch_count(ctx: Context) -> int:
 
 
 KERNEL_CLASSES = ("assign_main", "assign_prep", "resolve", "objective", "update_accum", "update_finish",
-                  "reshape", "decode", "other", "assign_finish", "update_delta")
+                  "reshape", "decode", "other", "assign_finish", "update_delta", "linear")
 
 
 def cc_profile_enable(ctx: Context, on: bool) -> None:
@@ -278,6 +287,52 @@ def cc_fit(ctx, X, N, g, K, iters, C, idx, dist, counts, objective_trace=None, s
                          _ptr(objective_trace), _stream(stream)), "cc_fit")
 
 
+def cc_set_empty_rule(ctx, rule: int) -> None:
+    _check(load().cc_set_empty_rule(ctx._h, rule), "cc_set_empty_rule")
+
+
+def cc_train_points(N: int, K: int, max_points_per_centroid: int) -> int:
+    return int(load().cc_train_points(N, K, max_points_per_centroid))
+
+
+def cc_fit_sampled(ctx, X, N, g, K, iters, max_points_per_centroid, seed, X_train, C, idx, dist, counts,
+                   objective_trace=None, stream=None) -> None:
+    _check(load().cc_fit_sampled(ctx._h, _ptr(X), N, g, K, iters, max_points_per_centroid, seed, _ptr(X_train), _ptr(C),
+                                 _ptr(idx), _ptr(dist), _ptr(counts), _ptr(objective_trace), _stream(stream)),
+           "cc_fit_sampled")
+
+
+def cc_quantize_codebook(ctx, C16, K, g, bits, q, scale, C16_dequantized=None, stream=None) -> None:
+    _check(load().cc_quantize_codebook(ctx._h, _ptr(C16), K, g, bits, _ptr(q), _ptr(scale), _ptr(C16_dequantized),
+                                       _stream(stream)), "cc_quantize_codebook")
+
+
+def cc_schedule_matrices(sizes, world: int, rank: int):
+    """Indices (increasing) of the matrices that fall to `rank` in the size-balanced split."""
+    n = len(sizes)
+    arr = (_i64 * max(n, 1))(*[int(v) for v in sizes])
+    mine = (ct.c_int32 * max(n, 1))()
+    cnt = ct.c_int32(0)
+    _check(load().cc_schedule_matrices(n, arr, world, rank, mine, ct.byref(cnt)), "cc_schedule_matrices")
+    return [int(mine[i]) for i in range(cnt.value)]
+
+
+def cc_compress_many(ctx, W_hosts, d_outs, d_ins, g, K, iters, seeds, layout, C16_hosts, idx_hosts,
+                     objective_trace_hosts=None, W_hat_hosts=None, stream=None) -> None:
+    """Lists of HOST tensors, one entry per matrix (entries of the two optional lists may be None)."""
+    n = len(W_hosts)
+
+    def ptrs(lst):
+        if lst is None:
+            return None
+        assert len(lst) == n and all(t is None or not t.is_cuda for t in lst)
+        return (_vp * max(n, 1))(*[_ptr(t) for t in lst])
+
+    _check(load().cc_compress_many(ctx._h, n, ptrs(W_hosts), (_i64 * max(n, 1))(*d_outs), (_i64 * max(n, 1))(*d_ins), g, K,
+                                   iters, (_u64 * max(n, 1))(*seeds), layout, ptrs(C16_hosts), ptrs(idx_hosts),
+                                   ptrs(objective_trace_hosts), ptrs(W_hat_hosts), _stream(stream)), "cc_compress_many")
+
+
 def cc_finalize(ctx, X, N, g, C, K, C16, idx, dist=None, objective=None, stream=None) -> None:
     _check(load().cc_finalize(ctx._h, _ptr(X), N, g, _ptr(C), K, _ptr(C16), _ptr(idx), _ptr(dist),
                               _ptr(objective), _stream(stream)), "cc_finalize")
@@ -286,6 +341,15 @@ def cc_finalize(ctx, X, N, g, C, K, C16, idx, dist=None, objective=None, stream=
 def cc_decode(ctx, C16, K, g, idx, d_out, d_in, layout, W_hat, stream=None) -> None:
     _check(load().cc_decode(ctx._h, _ptr(C16), K, g, _ptr(idx), d_out, d_in, layout, _ptr(W_hat),
                             _stream(stream)), "cc_decode")
+
+
+def cc_linear_workspace_bytes(ctx, M: int, d_out: int, d_in: int) -> int:
+    return int(load().cc_linear_workspace_bytes(ctx._h, M, d_out, d_in))
+
+
+def cc_linear_forward(ctx, x, M, C16, K, g, idx, d_out, d_in, bias, y, stream=None) -> None:
+    _check(load().cc_linear_forward(ctx._h, _ptr(x), M, _ptr(C16), K, g, _ptr(idx), d_out, d_in, _ptr(bias), _ptr(y),
+                                    _stream(stream)), "cc_linear_forward")
 
 
 def cc_poll_status(ctx, stream=None) -> None:

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 INCLUDE = os.path.join(os.path.dirname(HERE), "include")
 LIB = os.path.join(HERE, "libcluscomp.so")
-SOURCES = ["cc_api.cu", "cc_layout.cu", "cc_assign_ffma.cu", "cc_assign_tensor.cu", "cc_update.cu", "cc_measure.cu"]
+SOURCES = ["cc_api.cu", "cc_layout.cu", "cc_assign_ffma.cu", "cc_assign_tensor.cu", "cc_update.cu", "cc_measure.cu", "cc_linear.cu", "cc_extras.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "-I", INCLUDE, "-I", CSRC]
 

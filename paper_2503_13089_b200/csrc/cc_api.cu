@@ -57,6 +57,38 @@ inline uint64_t splitmix64(uint64_t& s) {
     return z ^ (z >> 31);
 }
 
+// The same shuffle for any number n <= N of positions, written to 32-bit words: with many positions
+// the whole array is kept, with few only the touched entries.
+bool partial_shuffle_u32(int64_t N, int64_t n, uint64_t seed, uint32_t* pos) {
+    uint64_t s = seed;
+    if (n * 8 >= N) {
+        std::vector<uint32_t> a;
+        try { a.resize((size_t)N); } catch (...) { return false; }
+        for (int64_t i = 0; i < N; ++i) a[(size_t)i] = (uint32_t)i;
+        for (int64_t i = 0; i < n; ++i) {
+            const int64_t j = i + (int64_t)(splitmix64(s) % (uint64_t)(N - i));
+            const uint32_t t = a[(size_t)i];
+            a[(size_t)i] = a[(size_t)j];
+            a[(size_t)j] = t;
+            pos[i] = a[(size_t)i];
+        }
+        return true;
+    }
+    std::unordered_map<int64_t, int64_t> moved;
+    moved.reserve((size_t)n * 2);
+    for (int64_t i = 0; i < n; ++i) {
+        const int64_t j = i + (int64_t)(splitmix64(s) % (uint64_t)(N - i));
+        auto itj = moved.find(j);
+        const int64_t vj = (itj == moved.end()) ? j : itj->second;
+        auto iti = moved.find(i);
+        const int64_t vi = (iti == moved.end()) ? i : iti->second;
+        moved[j] = vi;
+        moved[i] = vj;
+        pos[i] = (uint32_t)vj;
+    }
+    return true;
+}
+
 // Only the K touched entries of the shuffled array are kept (a map from position to content).
 void partial_shuffle(int64_t N, int K, uint64_t seed, int64_t* pos) {
     std::unordered_map<int64_t, int64_t> moved;
@@ -133,6 +165,7 @@ cc_status cc_create(cc_ctx** out, int device) {
     c->prof = nullptr;
     c->e2e_buf = nullptr;
     c->e2e_bytes = 0;
+    c->empty_rule = CC_EMPTY_KEEP;
     *out = c;
     return CC_OK;
 }
@@ -367,6 +400,105 @@ cc_status cc_fit(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, int K, int it
     return CC_OK;
 }
 
+cc_status cc_set_empty_rule(cc_ctx* ctx, int rule) {
+    if (!ctx) return CC_ERR_NULL;
+    if (rule != CC_EMPTY_KEEP && rule != CC_EMPTY_SPLIT_LARGEST) return CC_ERR_LAYOUT;
+    ctx->empty_rule = rule;
+    return CC_OK;
+}
+
+int64_t cc_train_points(int64_t N, int K, int max_points_per_centroid) {
+    if (N < 1 || K < 1 || K > 65536 || max_points_per_centroid < 1) return -1;
+    const int64_t n = (int64_t)max_points_per_centroid * K;
+    return n < N ? n : N;
+}
+
+cc_status cc_fit_sampled(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, int K, int iters, int max_points_per_centroid,
+                         uint64_t seed, uint16_t* X_train, float* C, uint16_t* idx, float* dist, int32_t* counts,
+                         double* objective_trace, void* stream) {
+    if (!ctx || !X || !C || !idx || !counts) return CC_ERR_NULL;
+    cc_status s = check_common(ctx, N, g, K, true);
+    if (s != CC_OK) return s;
+    if (N < 1 || iters < 0 || max_points_per_centroid < 1) return CC_ERR_SHAPE;
+    if (!aligned16(X) || !aligned16(C)) return CC_ERR_ALIGN;
+    const int64_t n = cc_train_points(N, K, max_points_per_centroid);
+    if (n < N && !X_train) return CC_ERR_NULL;
+    if (n < N && !aligned16(X_train)) return CC_ERR_ALIGN;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (n < N) {
+        std::vector<uint32_t> pos;
+        try { pos.resize((size_t)n); } catch (...) { return CC_ERR_CUDA; }
+        if (!partial_shuffle_u32(N, n, seed, pos.data())) return CC_ERR_CUDA;
+        const WsLayout L = cc_ws_layout(N, g, K);
+        unsigned* pos_dev = reinterpret_cast<unsigned*>(static_cast<char*>(ctx->ws) + L.flagged);   // free until the first E-step
+        // pageable source: the copy is staged before the call returns, so `pos` may go out of scope
+        if (cudaMemcpyAsync(pos_dev, pos.data(), sizeof(uint32_t) * (size_t)n, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return CC_ERR_CUDA;
+        if (cc_launch_gather_rows(ctx, X, g, pos_dev, n, X_train, st) != cudaSuccess) return CC_ERR_CUDA;
+        s = cc_fit(ctx, X_train, n, g, K, iters, C, idx, dist, counts, objective_trace, stream);
+    } else {
+        s = cc_fit(ctx, X, N, g, K, iters, C, idx, dist, counts, objective_trace, stream);
+    }
+    if (s != CC_OK) return s;
+    return cc_assign(ctx, X, N, g, C, K, idx, dist, nullptr, nullptr, stream);
+}
+
+cc_status cc_quantize_codebook(cc_ctx* ctx, const uint16_t* C16, int K, int g, int bits, uint8_t* q, float* scale,
+                               uint16_t* C16_dequantized, void* stream) {
+    if (!ctx || !C16 || !q || !scale) return CC_ERR_NULL;
+    if (g < 1 || g > 16) return CC_ERR_UNSUPPORTED_G;
+    if (K < 1 || K > 65536) return CC_ERR_K_RANGE;
+    if (bits != 8 && bits != 4) return CC_ERR_SHAPE;
+    if (!ctx->ws || ctx->ws_bytes < 256) return CC_ERR_WORKSPACE;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    return from_cuda(cc_launch_quantize_codebook(ctx, C16, (int64_t)K * g, bits, q, scale, C16_dequantized,
+                                                 (cudaStream_t)stream));
+}
+
+cc_status cc_schedule_matrices(int n, const int64_t* sizes_host, int world, int rank, int32_t* mine_host, int32_t* n_mine_host) {
+    if (!sizes_host || !mine_host || !n_mine_host) return CC_ERR_NULL;
+    if (n < 0 || world < 1 || rank < 0 || rank >= world) return CC_ERR_SHAPE;
+    // longest-processing-time first: matrices by decreasing size (lower index first among equals), each to
+    // the rank with the smallest load so far (lowest rank among equals)
+    std::vector<int> order((size_t)n);
+    for (int i = 0; i < n; ++i) order[(size_t)i] = i;
+    for (int i = 1; i < n; ++i) {                 // insertion sort: stable, n is a few hundred at most
+        const int v = order[(size_t)i];
+        int j = i - 1;
+        while (j >= 0 && sizes_host[order[(size_t)j]] < sizes_host[v]) { order[(size_t)j + 1] = order[(size_t)j]; --j; }
+        order[(size_t)j + 1] = v;
+    }
+    std::vector<int64_t> load((size_t)world, 0);
+    std::vector<char> is_mine((size_t)n, 0);
+    for (int k = 0; k < n; ++k) {
+        const int i = order[(size_t)k];
+        int r = 0;
+        for (int q = 1; q < world; ++q) if (load[(size_t)q] < load[(size_t)r]) r = q;
+        load[(size_t)r] += sizes_host[i];
+        if (r == rank) is_mine[(size_t)i] = 1;
+    }
+    int m = 0;
+    for (int i = 0; i < n; ++i) if (is_mine[(size_t)i]) mine_host[m++] = i;
+    *n_mine_host = m;
+    return CC_OK;
+}
+
+cc_status cc_compress_many(cc_ctx* ctx, int n, const uint16_t* const* W_hosts, const int64_t* d_outs, const int64_t* d_ins,
+                           int g, int K, int iters, const uint64_t* seeds, int layout, uint16_t* const* C16_hosts,
+                           uint16_t* const* idx_hosts, double* const* objective_trace_hosts, uint16_t* const* W_hat_hosts,
+                           void* stream) {
+    if (!ctx || !W_hosts || !d_outs || !d_ins || !seeds || !C16_hosts || !idx_hosts) return CC_ERR_NULL;
+    if (n < 0) return CC_ERR_SHAPE;
+    for (int i = 0; i < n; ++i) {
+        const cc_status s = cc_compress_host(ctx, W_hosts[i], d_outs[i], d_ins[i], g, K, iters, seeds[i], layout, C16_hosts[i],
+                                             idx_hosts[i], objective_trace_hosts ? objective_trace_hosts[i] : nullptr,
+                                             W_hat_hosts ? W_hat_hosts[i] : nullptr, stream);
+        if (s != CC_OK) return s;
+    }
+    return CC_OK;
+}
+
 cc_status cc_finalize(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, const float* C, int K, uint16_t* C16,
                       uint16_t* idx, float* dist, double* objective, void* stream) {
     if (!ctx || !X || !C || !C16 || !idx) return CC_ERR_NULL;
@@ -394,6 +526,25 @@ cc_status cc_decode(cc_ctx* ctx, const uint16_t* C16, int K, int g, const uint16
     if (!aligned16(C16) || !aligned16(W_hat)) return CC_ERR_ALIGN;
     if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
     return from_cuda(cc_launch_decode(ctx, C16, K, g, idx, d_out, d_in, layout, W_hat, (cudaStream_t)stream));
+}
+
+size_t cc_linear_workspace_bytes(cc_ctx* ctx, int64_t M, int64_t d_out, int64_t d_in) {
+    if (!ctx || M < 1 || d_out < 1 || d_in < 1 || M * d_out >= (int64_t)1 << 31 || d_in >= (int64_t)1 << 31) return 0;
+    return cc_linear_scratch_bytes(M, d_out, d_in, ctx->sm_count);
+}
+
+cc_status cc_linear_forward(cc_ctx* ctx, const uint16_t* x, int64_t M, const uint16_t* C16, int K, int g,
+                            const uint16_t* idx, int64_t d_out, int64_t d_in, const float* bias, float* y,
+                            void* stream) {
+    if (!ctx || !x || !C16 || !idx || !y) return CC_ERR_NULL;
+    if (g < 1 || g > 16) return CC_ERR_UNSUPPORTED_G;
+    if (K < 1 || K > 65536) return CC_ERR_K_RANGE;
+    const int64_t N = cc_num_subvectors(d_out, d_in, g, CC_LAYOUT_PAPER_T);
+    if (N < 1 || N >= (int64_t)1 << 31 || M < 1 || M * d_out >= (int64_t)1 << 31) return CC_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(C16) || !aligned16(y)) return CC_ERR_ALIGN;
+    if (!ctx->ws || ctx->ws_bytes < cc_linear_scratch_bytes(M, d_out, d_in, ctx->sm_count)) return CC_ERR_WORKSPACE;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    return from_cuda(cc_launch_linear_forward(ctx, x, M, C16, K, g, idx, d_out, d_in, bias, y, (cudaStream_t)stream));
 }
 
 cc_status cc_poll_status(cc_ctx* ctx, void* stream) {

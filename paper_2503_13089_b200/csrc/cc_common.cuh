@@ -14,7 +14,7 @@
 // Kernel classes for the optional per-kernel event timing (cc_profile_*).
 enum { CC_K_ASSIGN_MAIN = 0, CC_K_ASSIGN_PREP = 1, CC_K_RESOLVE = 2, CC_K_OBJECTIVE = 3, CC_K_UPDATE_ACCUM = 4,
        CC_K_UPDATE_FINISH = 5, CC_K_RESHAPE = 6, CC_K_DECODE = 7, CC_K_OTHER = 8, CC_K_ASSIGN_FINISH = 9, CC_K_UPDATE_DELTA = 10,
-       CC_K_COUNT = 11 };
+       CC_K_LINEAR = 11, CC_K_COUNT = 12 };
 constexpr int CC_PROF_CAP = 8192;
 
 struct cc_prof_slot { cudaEvent_t a, b; int kind; };
@@ -33,6 +33,7 @@ struct cc_ctx {
     cc_prof_slot* prof;   // CC_PROF_CAP slots, events created on first use
     void* e2e_buf;        // device memory of cc_compress_host, grown on demand, freed by cc_destroy
     size_t e2e_bytes;
+    int empty_rule;       // CC_EMPTY_*
 };
 
 // Brackets one kernel launch with events on its stream when timing is enabled, and counts it.
@@ -118,6 +119,18 @@ cudaError_t cc_launch_tensor_finish_only(cc_ctx*, const WsLayout&, const uint16_
 cudaError_t cc_launch_assign_tail(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const float* C,
                                   int K, uint16_t* idx, float* dist, double* objective, int64_t* n_resolved,
                                   cudaStream_t);
+
+// Compressed linear layer: y = x . decode(C16, idx)^T (+ bias), the decoded weight never stored.
+size_t cc_linear_scratch_bytes(int64_t M, int64_t d_out, int64_t d_in, int sm_count);
+cudaError_t cc_launch_linear_forward(cc_ctx*, const uint16_t* x, int64_t M, const uint16_t* C16, int K, int g,
+                                     const uint16_t* idx, int64_t d_out, int64_t d_in, const float* bias, float* y,
+                                     cudaStream_t);
+
+cudaError_t cc_launch_quantize_codebook(cc_ctx*, const uint16_t* C16, int64_t n, int bits, uint8_t* q, float* scale,
+                                        uint16_t* deq, cudaStream_t);
+cudaError_t cc_launch_gather_rows(cc_ctx*, const uint16_t* X, int g, const unsigned* pos_dev, int64_t n, uint16_t* out,
+                                  cudaStream_t);
+cudaError_t cc_launch_split_empty(cc_ctx*, const WsLayout&, float* C, int K, int g, const int32_t* counts, cudaStream_t);
 
 cudaError_t cc_launch_update(cc_ctx*, const WsLayout&, const uint16_t* X, int64_t N, int g, const uint16_t* idx,
                              int K, float* C, int32_t* counts, cudaStream_t);

@@ -1,0 +1,344 @@
+// Forward of the compressed linear layer (appendix listing): out = x . weight (+ bias) with
+// weight = codebook[code] viewed as (in_features, out_features + pad), the padded columns dropped.
+// The decoded weight is never written to memory: the kernel gathers codebook rows straight into the
+// shared-memory operand of a tcgen05 GEMM.
+//
+// The product is computed transposed, out^T = weight^T . x^T, so that the WEIGHT is the 128-row
+// operand of the MMA (128 out_features per CTA) and the tokens are its N dimension (16..256 columns,
+// FP32 accumulators in TMEM).  A batch of a few tokens then costs a narrow MMA instead of a padded
+// 128-row one, and the weight -- the large operand -- is gathered exactly once per token block.
+//
+// Per stage of 64 in_features the producer warps build
+//   A: 128 out_features x 64 in_features, FP16, canonical K-major layout without swizzle.  One work
+//      item = 8 consecutive in_features x one code group (g consecutive out_features): 8 codes, 8
+//      codebook rows, transposed in registers into g rows of 16 bytes.
+//   B: NT tokens x 64 in_features of x (16-byte copies).
+// A ring of STAGES such stages feeds one MMA-issuing thread (4 MMAs of K = 16 per stage); full / empty
+// mbarriers, every wait bounded by a clock limit (a wait that runs out raises CC_DEV_TIMEOUT, the
+// CTA stops issuing work, skips its stores and still frees its tensor memory).
+// With few tokens and few 128-row tiles the in_features are split across CTAs (split-K): every split
+// writes its partial sums to scratch and a second kernel adds them in a fixed order, so the result
+// does not depend on scheduling.
+#include <cuda_fp16.h>
+
+#include "cc_common.cuh"
+#include "cc_tcgen05.cuh"
+
+namespace {
+
+constexpr int LM = 128;                 // out_features per CTA = MMA M = TMEM lanes
+constexpr int LKB = 64;                 // in_features per pipeline stage
+constexpr int LSTAGES = 4;
+constexpr int LPROD = 256;              // producer threads (8 warps); warps 0..3 also run the epilogue
+constexpr int LTHREADS = LPROD + 32;    // + the MMA warp
+constexpr int LNT_MAX = 256;            // tokens per CTA = MMA N
+constexpr int A_STAGE = LM * LKB * 2;   // bytes
+
+// Row of G halves of the codebook as raw bit patterns.
+template <int G>
+__device__ __forceinline__ void load_code_row(const uint16_t* __restrict__ C16, int code, uint16_t* h) {
+    const uint16_t* row = C16 + (int64_t)code * G;
+    if constexpr (G % 8 == 0) {
+#pragma unroll
+        for (int v = 0; v < G / 8; ++v) {
+            const uint4 u = __ldg(reinterpret_cast<const uint4*>(row) + v);
+            const unsigned w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+            for (int k = 0; k < 4; ++k) { h[v * 8 + 2 * k] = w[k] & 0xffffu; h[v * 8 + 2 * k + 1] = w[k] >> 16; }
+        }
+    } else if constexpr (G % 4 == 0) {
+#pragma unroll
+        for (int v = 0; v < G / 4; ++v) {
+            const uint2 u = __ldg(reinterpret_cast<const uint2*>(row) + v);
+            h[v * 4] = u.x & 0xffffu; h[v * 4 + 1] = u.x >> 16; h[v * 4 + 2] = u.y & 0xffffu; h[v * 4 + 3] = u.y >> 16;
+        }
+    } else if constexpr (G % 2 == 0) {
+#pragma unroll
+        for (int v = 0; v < G / 2; ++v) {
+            const unsigned u = __ldg(reinterpret_cast<const unsigned*>(row) + v);
+            h[v * 2] = u & 0xffffu; h[v * 2 + 1] = u >> 16;
+        }
+    } else {
+#pragma unroll
+        for (int t = 0; t < G; ++t) h[t] = __ldg(row + t);
+    }
+}
+
+// blockIdx.x: tile of 128 out_features; blockIdx.y: block of NT tokens; blockIdx.z: split of the
+// in_features (chunks_per_split stages each).  out: y itself (splits == 1) or this split's slab of
+// partial sums, both M x d_out FP32 row-major.
+template <int G>
+__global__ void __launch_bounds__(LTHREADS, 1)
+linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __restrict__ C16,
+                      const uint16_t* __restrict__ idx, int d_out, int d_in, int out_groups, int NT,
+                      int tmem_cols, int chunks_per_split, float* __restrict__ out, int64_t split_stride,
+                      const float* __restrict__ bias, unsigned* __restrict__ status) {
+    extern __shared__ __align__(1024) unsigned char smem_raw[];
+    const int b_stage = NT * LKB * 2;
+    unsigned char* sA = smem_raw;                                   // LSTAGES tiles of 128 x 64
+    unsigned char* sB = sA + LSTAGES * A_STAGE;                     // LSTAGES tiles of NT x 64
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sB + LSTAGES * b_stage);
+    uint64_t* full = bars, *empty = bars + LSTAGES, *acc_full = bars + 2 * LSTAGES;
+    uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * LSTAGES + 1);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int o0 = blockIdx.x * LM;
+    const int m0 = blockIdx.y * NT;
+    const int n_chunks_total = (d_in + LKB - 1) / LKB;
+    const int chunk_first = blockIdx.z * chunks_per_split;
+    int n_chunks = n_chunks_total - chunk_first;
+    n_chunks = n_chunks < chunks_per_split ? n_chunks : chunks_per_split;
+    if (n_chunks < 0) n_chunks = 0;
+
+    if (tid == 0) {
+        for (int s = 0; s < LSTAGES; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(full + s)), "r"(LPROD));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(empty + s)));
+        }
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(acc_full)));
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 0) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
+                     "r"(tmem_cols));
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp < LPROD / 32) {
+        // ------------------------------------------------------------ producers
+        // code groups that touch this tile of out_features
+        const int grp_lo = o0 / G;
+        int grp_hi = (o0 + LM - 1) / G;
+        if (grp_hi > out_groups - 1) grp_hi = out_groups - 1;
+        const int n_grp = grp_hi - grp_lo + 1;                      // >= 1: o0 < d_out <= out_groups * G
+        const bool vec_x = (d_in % 8) == 0;
+        bool ok = true;
+        for (int c = 0; c < n_chunks && ok; ++c) {
+            const int st = c % LSTAGES;
+            ok = mbar_wait(smem_u32(empty + st), ((c / LSTAGES) & 1) ^ 1, abort_flag);
+            if (!ok) break;
+            unsigned char* tA = sA + st * A_STAGE;
+            unsigned char* tB = sB + st * b_stage;
+            const int i0 = (chunk_first + c) * LKB;
+            // ---- A: gather, transpose, store.  item = (block of 8 in_features, code group)
+            for (int item = tid; item < (LKB / 8) * n_grp; item += LPROD) {
+                const int ib = item / n_grp, gl = item - ib * n_grp;
+                const int grp = grp_lo + gl;
+                uint16_t v[8][G];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int i = i0 + ib * 8 + u;
+                    if (i < d_in) {
+                        const int code = __ldg(idx + (int64_t)i * out_groups + grp);
+                        load_code_row<G>(C16, code, v[u]);
+                    } else {
+#pragma unroll
+                        for (int t = 0; t < G; ++t) v[u][t] = 0;
+                    }
+                }
+#pragma unroll
+                for (int t = 0; t < G; ++t) {
+                    const int r = grp * G + t - o0;                 // row of the tile = out_feature - o0
+                    if (r < 0 || r >= LM) continue;
+                    uint4 w;
+                    w.x = (unsigned)v[0][t] | ((unsigned)v[1][t] << 16);
+                    w.y = (unsigned)v[2][t] | ((unsigned)v[3][t] << 16);
+                    w.z = (unsigned)v[4][t] | ((unsigned)v[5][t] << 16);
+                    w.w = (unsigned)v[6][t] | ((unsigned)v[7][t] << 16);
+                    *reinterpret_cast<uint4*>(tA + canon_bytes(r, ib * 8, LM)) = w;
+                }
+            }
+            // ---- B: the tokens' slice of x, 8 in_features (16 bytes) at a time
+            for (int item = tid; item < NT * (LKB / 8); item += LPROD) {
+                const int kc = item % (LKB / 8), r = item / (LKB / 8);
+                const int m = m0 + r, i = i0 + kc * 8;
+                uint4 w = make_uint4(0u, 0u, 0u, 0u);
+                if (m < M && i < d_in) {
+                    const uint16_t* src = x + (int64_t)m * d_in + i;
+                    if (vec_x) {
+                        w = __ldg(reinterpret_cast<const uint4*>(src));
+                    } else {
+                        unsigned short h[8];
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) h[u] = (i + u < d_in) ? __ldg(src + u) : (unsigned short)0;
+                        w.x = (unsigned)h[0] | ((unsigned)h[1] << 16);
+                        w.y = (unsigned)h[2] | ((unsigned)h[3] << 16);
+                        w.z = (unsigned)h[4] | ((unsigned)h[5] << 16);
+                        w.w = (unsigned)h[6] | ((unsigned)h[7] << 16);
+                    }
+                }
+                *reinterpret_cast<uint4*>(tB + canon_bytes(r, kc * 8, NT)) = w;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> async proxy (MMA)
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(full + st)) : "memory");
+        }
+        // ------------------------------------------------------------ epilogue (warps 0..3)
+        if (warp < 4) {
+            ok = ok && mbar_wait(smem_u32(acc_full), 0, abort_flag);
+            asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+            const int o = o0 + warp * 32 + lane;                    // TMEM lane = out_feature of the tile
+            float* dst = out + (int64_t)blockIdx.z * split_stride;
+            const float b = (bias && o < d_out) ? __ldg(bias + o) : 0.f;
+            for (int cb = 0; cb < NT; cb += 32) {
+                uint32_t v[32];
+                TMEM_LD32(v, tmem + ((uint32_t)(warp * 32) << 16) + cb);
+                TMEM_WAIT32(v);
+                if (ok && !*abort_flag && o < d_out) {
+#pragma unroll
+                    for (int u = 0; u < 32; ++u) {
+                        const int m = m0 + cb + u;
+                        if (cb + u < NT && m < M)                   // 32 lanes write 32 consecutive out_features
+                            dst[(int64_t)m * d_out + o] = (n_chunks > 0 ? __uint_as_float(v[u]) : 0.f) + b;
+                    }
+                }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------ MMA warp: one thread issues
+        if (lane == 0) {
+            // kind::f16: D = F32 (bits 4-5 = 1), A = B = F16 (0), both K-major, N >> 3 at bit 17, M >> 4 at bit 24
+            const uint32_t idesc = (1u << 4) | ((uint32_t)(NT >> 3) << 17) | ((uint32_t)(LM >> 4) << 24);
+            const uint64_t descA0 = make_desc(smem_u32(sA), LM * 16, 128);
+            const uint64_t descB0 = make_desc(smem_u32(sB), NT * 16, 128);
+            bool ok = true;
+            for (int c = 0; c < n_chunks && ok; ++c) {
+                const int st = c % LSTAGES;
+                ok = mbar_wait(smem_u32(full + st), (c / LSTAGES) & 1, abort_flag);
+                if (!ok) break;
+                asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+                const uint64_t descA = descA0 + (uint64_t)((st * A_STAGE) >> 4);
+                const uint64_t descB = descB0 + (uint64_t)((st * b_stage) >> 4);
+#pragma unroll
+                for (int s = 0; s < LKB / 16; ++s) {
+                    const uint64_t da = descA + (uint64_t)((s * 2 * (LM * 16)) >> 4);
+                    const uint64_t db = descB + (uint64_t)((s * 2 * (NT * 16)) >> 4);
+                    const uint32_t acc = (c > 0 || s > 0) ? 1u : 0u;
+                    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                                 ::"r"(tmem), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+                }
+                // the stage may be refilled once these MMAs have read it
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                             ::"r"(smem_u32(empty + st)) : "memory");
+            }
+            if (ok)
+                asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
+                             ::"r"(smem_u32(acc_full)) : "memory");
+            else
+                *abort_flag = 1;   // the epilogue's wait on acc_full returns at its next look at the flag
+        }
+    }
+    if (*abort_flag && lane == 0) atomicOr(status, CC_DEV_TIMEOUT);
+    asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
+    __syncthreads();
+    if (warp == 0)
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"(tmem_cols));
+}
+
+// y[m][o] = bias[o] + sum over the splits, in split order.
+__global__ void __launch_bounds__(256)
+linear_reduce_kernel(const float* __restrict__ partial, int splits, int64_t n, int d_out, const float* __restrict__ bias,
+                     float* __restrict__ y) {
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x) {
+        float s = bias ? __ldg(bias + (int)(e % d_out)) : 0.f;
+        for (int k = 0; k < splits; ++k) s += partial[(int64_t)k * n + e];
+        y[e] = s;
+    }
+}
+
+struct LinearPlan { int NT, tmem_cols, o_tiles, tok_blocks, splits, chunks_per_split; size_t smem; };
+
+LinearPlan linear_plan(int64_t M, int64_t d_out, int64_t d_in, int sm_count) {
+    LinearPlan p;
+    const int64_t mt = M < LNT_MAX ? M : LNT_MAX;
+    p.NT = (int)((mt + 15) / 16 * 16);
+    p.tmem_cols = 32;
+    while (p.tmem_cols < p.NT) p.tmem_cols *= 2;
+    p.o_tiles = (int)((d_out + LM - 1) / LM);
+    p.tok_blocks = (int)((M + p.NT - 1) / p.NT);
+    const int chunks = (int)((d_in + LKB - 1) / LKB);
+    int splits = sm_count / (p.o_tiles * p.tok_blocks);             // fill the SMs when there are few tiles
+    if (splits > chunks / 4) splits = chunks / 4;                   // at least four stages of work per CTA
+    if (splits < 1) splits = 1;
+    p.chunks_per_split = (chunks + splits - 1) / splits;
+    p.splits = (chunks + p.chunks_per_split - 1) / p.chunks_per_split;
+    p.smem = (size_t)LSTAGES * (A_STAGE + (size_t)p.NT * LKB * 2) + 256;
+    return p;
+}
+
+}  // namespace
+
+size_t cc_linear_scratch_bytes(int64_t M, int64_t d_out, int64_t d_in, int sm_count) {
+    const LinearPlan p = linear_plan(M, d_out, d_in, sm_count);
+    return 256 + (p.splits > 1 ? (size_t)p.splits * (size_t)M * (size_t)d_out * 4 : 0);
+}
+
+#define CC_LINEAR_DISPATCH(g, CALL)                                                                 \
+    switch (g) {                                                                                    \
+        case 1: CALL(1); break;   case 2: CALL(2); break;   case 3: CALL(3); break;                 \
+        case 4: CALL(4); break;   case 5: CALL(5); break;   case 6: CALL(6); break;                 \
+        case 7: CALL(7); break;   case 8: CALL(8); break;   case 9: CALL(9); break;                 \
+        case 10: CALL(10); break; case 11: CALL(11); break; case 12: CALL(12); break;               \
+        case 13: CALL(13); break; case 14: CALL(14); break; case 15: CALL(15); break;               \
+        case 16: CALL(16); break;                                                                   \
+        default: return cudaErrorInvalidValue;                                                      \
+    }
+
+namespace {
+
+template <int G>
+cudaError_t launch_linear(cc_ctx* ctx, const LinearPlan& p, const uint16_t* x, int M, const uint16_t* C16,
+                          const uint16_t* idx, int d_out, int d_in, int out_groups, float* out, int64_t split_stride,
+                          const float* bias, unsigned* status, cudaStream_t st) {
+    static size_t attr_dev[64] = {};
+    size_t& have = attr_dev[ctx->device & 63];
+    if (have < p.smem) {
+        const cudaError_t e = cudaFuncSetAttribute(linear_forward_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)(LSTAGES * (A_STAGE + LNT_MAX * LKB * 2) + 256));
+        if (e != cudaSuccess) return e;
+        have = LSTAGES * (A_STAGE + LNT_MAX * LKB * 2) + 256;
+    }
+    const dim3 grid(p.o_tiles, p.tok_blocks, p.splits);
+    linear_forward_kernel<G><<<grid, LTHREADS, p.smem, st>>>(x, M, C16, idx, d_out, d_in, out_groups, p.NT, p.tmem_cols,
+                                                             p.chunks_per_split, out, split_stride, bias, status);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t cc_launch_linear_forward(cc_ctx* ctx, const uint16_t* x, int64_t M, const uint16_t* C16, int K, int g,
+                                     const uint16_t* idx, int64_t d_out, int64_t d_in, const float* bias, float* y,
+                                     cudaStream_t st) {
+    (void)K;
+    const LinearPlan p = linear_plan(M, d_out, d_in, ctx->sm_count);
+    char* ws = static_cast<char*>(ctx->ws);
+    unsigned* status = reinterpret_cast<unsigned*>(ws);
+    float* partial = reinterpret_cast<float*>(ws + 256);
+    const int out_groups = (int)((d_out + g - 1) / g);
+    const int64_t n = M * d_out;
+    cudaError_t e = cudaSuccess;
+    {
+        ProfScope ps(ctx, CC_K_LINEAR, st);
+        float* out = p.splits > 1 ? partial : y;
+        const float* b = p.splits > 1 ? nullptr : bias;
+#define CALL(G) e = launch_linear<G>(ctx, p, x, (int)M, C16, idx, (int)d_out, (int)d_in, out_groups, out, n, b, status, st)
+        CC_LINEAR_DISPATCH(g, CALL)
+#undef CALL
+    }
+    if (e != cudaSuccess) return e;
+    if (p.splits > 1) {
+        ProfScope ps(ctx, CC_K_LINEAR, st);
+        int64_t blocks = (n + 255) / 256;
+        const int64_t cap = (int64_t)ctx->sm_count * 8;
+        if (blocks > cap) blocks = cap;
+        linear_reduce_kernel<<<(unsigned)blocks, 256, 0, st>>>(partial, p.splits, n, (int)d_out, bias, y);
+        e = cudaGetLastError();
+    }
+    return e;
+}

@@ -188,10 +188,13 @@ cudaError_t cc_launch_update(cc_ctx* ctx, const WsLayout& L, const uint16_t* X, 
     int32_t* count_copies = nullptr;
     const cudaError_t e = accumulate_all(ctx, L, X, N, g, idx, K, counts, R, &count_copies, st);
     if (e != cudaSuccess) return e;
-    ProfScope ps(ctx, CC_K_UPDATE_FINISH, st);
-    update_finish_kernel<<<(K * g + 255) / 256, 256, 0, st>>>(reinterpret_cast<long long*>(ws + L.sum_lo),
-                                                             reinterpret_cast<long long*>(ws + L.sum_hi),
-                                                             count_copies, counts, K, g, R, C);
+    {
+        ProfScope ps(ctx, CC_K_UPDATE_FINISH, st);
+        update_finish_kernel<<<(K * g + 255) / 256, 256, 0, st>>>(reinterpret_cast<long long*>(ws + L.sum_lo),
+                                                                 reinterpret_cast<long long*>(ws + L.sum_hi),
+                                                                 count_copies, counts, K, g, R, C);
+    }
+    if (ctx->empty_rule == CC_EMPTY_SPLIT_LARGEST) return cc_launch_split_empty(ctx, L, C, K, g, counts, st);
     return cudaGetLastError();
 }
 
@@ -228,10 +231,13 @@ cudaError_t cc_launch_update_delta(cc_ctx* ctx, const WsLayout& L, const uint16_
         CC_UPDATE_DISPATCH(g, CALL)
 #undef CALL
     }
-    ProfScope ps(ctx, CC_K_UPDATE_FINISH, st);
-    update_finish_kernel<<<(K * g + 255) / 256, 256, 0, st>>>(reinterpret_cast<long long*>(sum_lo),
-                                                             reinterpret_cast<long long*>(sum_hi), counts, counts, K, g,
-                                                             1, C);
+    {
+        ProfScope ps(ctx, CC_K_UPDATE_FINISH, st);
+        update_finish_kernel<<<(K * g + 255) / 256, 256, 0, st>>>(reinterpret_cast<long long*>(sum_lo),
+                                                                 reinterpret_cast<long long*>(sum_hi), counts, counts, K,
+                                                                 g, 1, C);
+    }
+    if (ctx->empty_rule == CC_EMPTY_SPLIT_LARGEST) return cc_launch_split_empty(ctx, L, C, K, g, counts, st);
     return cudaGetLastError();
 }
 

@@ -78,3 +78,26 @@ def test_workload_sizes_follow_the_padding_rule():
             assert 1 <= w.K <= 65536 and n >= w.K
             padded += m.d_out % w.g != 0
     assert padded >= 4
+
+
+def test_schedule_matrices_is_the_size_balanced_split():
+    """Longest-processing-time first, as documented in the header.  One 7B decoder layer over two ranks,
+    worked out by hand: the three MLP matrices (2.8 M sub-vectors) go first -- rank 0, rank 1, rank 0 (equal
+    loads: the lower rank) -- then the four attention matrices (1.05 M) go to rank 1 three times (3.9, 4.9,
+    6.0 M against 5.6 M) and the last one to rank 0.  The Python helper of the multi-process tests states
+    the same rule and must agree on random sizes."""
+    from paper_2503_13089_b200 import sharding
+    att, mlp = 1048576, 2818048
+    sizes = [att, att, att, att, mlp, mlp, mlp]
+    assert cc.cc_schedule_matrices(sizes, 2, 0) == [3, 4, 6]
+    assert cc.cc_schedule_matrices(sizes, 2, 1) == [0, 1, 2, 5]
+    rng = np.random.default_rng(0)
+    for world in (1, 2, 3, 8):
+        for n in (0, 1, 5, 40):
+            sz = [int(v) for v in rng.integers(1, 1000, n)]
+            want = sharding.assign_matrices(sz, world)
+            got = [cc.cc_schedule_matrices(sz, world, r) for r in range(world)]
+            assert got == want
+            assert sorted(i for part in got for i in part) == list(range(n))
+    with pytest.raises(cc.CCError):
+        cc.cc_schedule_matrices([1, 2], 2, 2)

@@ -1,0 +1,94 @@
+"""GPU parity of the compressed linear layer's forward (appendix listing): y = x . codebook[code]-as-weight + bias
+through the C ABI against the float64 oracle, element by element.
+
+Tolerance: FP16 inputs are exact, their products are exact in FP32, and the only error is the FP32
+accumulation over d_in terms on the tensor core; 1e-3 relative, with an absolute floor of 1e-3 of the
+output's root mean square for outputs that cancel to (almost) zero.
+"""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+
+pytestmark = pytest.mark.gpu
+
+RTOL = 1e-3
+
+
+def _case(M, d_out, d_in, g, K, seed):
+    rng = np.random.default_rng(seed)
+    x = (rng.standard_normal((M, d_in)) * 0.5).astype(np.float16)
+    C16 = (rng.standard_t(3.0, (K, g)) * 0.02).astype(np.float16)
+    idx = rng.integers(0, K, oracle.num_subvectors(d_out, d_in, g)).astype(np.uint16)
+    bias = rng.standard_normal(d_out).astype(np.float32)
+    return x, C16, idx, bias
+
+
+def _gpu_forward(x, C16, idx, d_out, d_in, bias):
+    from paper_2503_13089_b200 import binding as cc
+    from tests import gpu_util as u
+    M = x.shape[0]
+    K, g = C16.shape
+    c = u.ctx()
+    c.ensure_workspace(len(idx), g, K, at_least=cc.cc_linear_workspace_bytes(c, M, d_out, d_in))
+    y = torch.full((M, d_out), float("nan"), dtype=torch.float32, device="cuda")
+    cc.cc_linear_forward(c, u.half_dev(x), M, u.half_dev(C16), K, g, u.dev(idx.view(np.int16)).view(torch.uint16),
+                         d_out, d_in, None if bias is None else u.dev(bias), y)
+    cc.cc_poll_status(c)
+    return y.cpu().numpy()
+
+
+def _check(y, want):
+    assert np.isfinite(y).all()
+    err = np.abs(y.astype(np.float64) - want)
+    bound = RTOL * np.abs(want) + RTOL * np.sqrt(np.mean(want ** 2))
+    assert np.all(err <= bound), "worst error / bound: %.3g" % float((err / bound).max())
+    return float((err / bound).max())
+
+
+@pytest.mark.parametrize("M,d_out,d_in,g,K", [
+    (1, 256, 512, 4, 256),          # one token: 16-column MMA, split over the in_features
+    (16, 1000, 520, 4, 700),        # ragged last tile of out_features; in_features not a multiple of 64
+    (5, 130, 67, 6, 50),            # padded out_features (130 = 21 x 6 + 4), in_features not a multiple of 8
+    (7, 75, 40, 9, 33), (3, 64, 24, 1, 5), (9, 96, 72, 3, 40), (20, 250, 128, 5, 90), (11, 260, 64, 7, 300),
+    (256, 512, 1024, 8, 4096),      # a full 256-token block
+    (300, 384, 256, 16, 1000),      # two token blocks, the second ragged
+    (130, 144, 328, 12, 77), (40, 280, 200, 10, 64), (33, 208, 136, 13, 21), (18, 300, 96, 14, 19),
+    (24, 330, 80, 15, 23), (12, 132, 88, 11, 17), (50, 136, 4104, 2, 9),
+    (64, 4096, 4096, 4, 65536),     # a 7B attention projection with the paper's largest codebook
+])
+def test_linear_forward_matches_oracle(M, d_out, d_in, g, K):
+    x, C16, idx, bias = _case(M, d_out, d_in, g, K, M + d_out + d_in + g)
+    want = oracle.linear_forward(x, C16, idx.astype(np.int32), d_out, d_in, bias)
+    y = _gpu_forward(x, C16, idx, d_out, d_in, bias)
+    worst = _check(y, want)
+    y2 = _gpu_forward(x, C16, idx, d_out, d_in, bias)
+    assert np.array_equal(y.view(np.uint32), y2.view(np.uint32))            # same bits on every call
+    y0 = _gpu_forward(x, C16, idx, d_out, d_in, None)                       # without bias
+    _check(y0, want - bias.astype(np.float64))
+    print("M=%d %dx%d g=%d K=%d: worst error %.3f of the bound" % (M, d_out, d_in, g, K, worst))
+
+
+def test_linear_forward_many_tokens_sampled_rows():
+    """4096 tokens through a 4096 x 4096 layer (g = 4, K = 65536): the oracle computes a seeded sample of the rows."""
+    M, d_out, d_in, g, K = 4096, 4096, 4096, 4, 65536
+    x, C16, idx, bias = _case(M, d_out, d_in, g, K, 5)
+    y = _gpu_forward(x, C16, idx, d_out, d_in, bias)
+    rows = np.sort(np.random.default_rng(6).choice(M, 12, replace=False))
+    want = oracle.linear_forward(np.ascontiguousarray(x[rows]), C16, idx.astype(np.int32), d_out, d_in, bias)
+    _check(y[rows], want)
+    assert np.isfinite(y).all()
+
+
+def test_linear_forward_equals_decode_then_matmul():
+    """The fused kernel against the unfused route on the GPU itself: cc_decode, then a float64 product on the host."""
+    from paper_2503_13089_b200 import binding as cc
+    from tests import gpu_util as u
+    M, d_out, d_in, g, K = 32, 520, 384, 8, 3000
+    x, C16, idx, bias = _case(M, d_out, d_in, g, K, 11)
+    y = _gpu_forward(x, C16, idx, d_out, d_in, None)
+    What = torch.zeros((d_out, d_in), dtype=torch.float16, device="cuda")
+    cc.cc_decode(u.ctx(), u.half_dev(C16), K, g, u.dev(idx.view(np.int16)).view(torch.uint16), d_out, d_in, 0, What)
+    W_hat = What.cpu().numpy().astype(np.float64)
+    _check(y, x.astype(np.float64) @ W_hat.T)

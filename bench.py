@@ -363,6 +363,42 @@ def summarise(w, Ns, phases, prof_steps, peaks, ceiling_scores, path):
     return out
 
 
+def linear_rows(cc, torch, ctx, peaks):
+    """Forward of the compressed linear layer (decode fused into the GEMM) on a 4096 x 4096 layer with the
+    paper's g = 4 / 65536-entry codebook, for 1 to 4096 tokens: time per call, tensor and HBM fractions."""
+    d_out = d_in = 4096
+    g, K = 4, 65536
+    N = d_in * d_out // g
+    gen = torch.Generator(device="cuda").manual_seed(1)
+    C16 = (torch.randn((K, g), device="cuda", generator=gen) * 0.02).to(torch.float16)
+    idx = torch.randint(-32768, 32768, (N,), device="cuda", generator=gen, dtype=torch.int16).view(torch.uint16)   # all 65536 codes
+    rows = []
+    for M in (1, 16, 256, 4096):
+        x = (torch.randn((M, d_in), device="cuda", generator=gen) * 0.5).to(torch.float16)
+        y = torch.empty((M, d_out), dtype=torch.float32, device="cuda")
+        ctx.ensure_workspace(N, g, K, at_least=cc.cc_linear_workspace_bytes(ctx, M, d_out, d_in))
+        for _ in range(3):
+            cc.cc_linear_forward(ctx, x, M, C16, K, g, idx, d_out, d_in, None, y)
+        reps = 20
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        a.record(torch.cuda.current_stream())
+        for _ in range(reps):
+            cc.cc_linear_forward(ctx, x, M, C16, K, g, idx, d_out, d_in, None, y)
+        b.record(torch.cuda.current_stream())
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / reps
+        flops = 2.0 * M * d_in * d_out
+        by = 2.0 * N + 2.0 * K * g + 2.0 * M * d_in + 4.0 * M * d_out          # codes, codebook, x, y
+        rows.append({"M": M, "d_out": d_out, "d_in": d_in, "g": g, "K": K, "ms": ms,
+                     "tflops": flops / (ms * 1e-3) / 1e12, "tensor_frac_of_measured_bf16": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
+                     "algorithmic_GBs": by / (ms * 1e-3) / 1e9, "frac_of_hbm": by / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                     "bytes_fused": by, "bytes_decode_then_gemm": by + 2 * 2.0 * d_in * d_out,
+                     "l2": "not flushed between the repetitions: codes (8 MB) and codebook (0.5 MB) stay in L2"})
+    cc.cc_poll_status(ctx)
+    return rows
+
+
 def run_kernel_mode(a):
     """One entry point, a few repetitions, per-kernel-class device times (CUDA events on the stream)."""
     import torch
@@ -599,6 +635,8 @@ def main():
                 del r2
                 torch.cuda.empty_cache()
 
+        linear = linear_rows(cc, torch, ctx, peaks) if (world == 1 and not args.no_secondary) else []
+
         cpu_baseline = None
         if not args.no_cpu_baseline and world == 1:
             import oracle
@@ -642,6 +680,7 @@ def main():
             "hbm_kernels": summ["hbm_kernels"],
             "kernels": summ["kernel_classes"],
             "workloads": others,
+            "linear_forward": linear,
             "peaks": peaks,
             "probes": {"min_rate_lane_instr_per_clk_per_sm": min_rate, "probe_sm_mhz": probe_mhz,
                        "probe_distinct_sms": probe_sms, "fp32_fma_tflops_scalar": fp32_scalar,

@@ -764,8 +764,9 @@ assign_tensor_persistent_kernel(const uint16_t* __restrict__ X, int64_t N, const
 // (sub, mul, add in dimension order, no contraction), the near-tie test and the stores.  A scan whose scores are off by at most
 //     E = ERR_UNITS 2^-24 (2||c||^2 + ||x||^2) + 2^-14 ||x||_1 / S + 2^-26 / S   (2^(e-25) / S with two norm pieces)
 // (|x_t| counted as at least 2^-14) may misorder two scores closer than 2E; every centroid at
-// least as close as the winner has 2||c||^2 + ||x||^2 <= 5||x||^2 + 4 d^2, so a point whose two
-// smallest scores are closer than 2E with that substitution goes to the exact stage.
+// least as close as the winner (distance d) has ||c|| <= ||x|| + d, hence 2||c||^2 + ||x||^2 <=
+// 3||x||^2 + 4||x|| d + 2 d^2, so a point whose two smallest scores are closer than 2E with that
+// substitution goes to the exact stage.
 template <int G>
 __global__ void __launch_bounds__(256)
 finish_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __restrict__ C, int K, int n_chunks,
@@ -867,7 +868,10 @@ finish_tensor_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __r
             idx[i] = (uint16_t)j1;
             dist[i] = (float)D;
             // A and L1 only feed the bound: FP32 is enough once they are rounded up a little
-            const double bound = 2.0 * ((double)TcCfg<G>::ERR_UNITS * 5.9604644775390625e-8 * (5.0 * (double)A * 1.0001 + 4.0 * D)
+            // 2||c||^2 + ||x||^2 <= 2 (||x|| + d)^2 + ||x||^2 = 3||x||^2 + 4||x|| d + 2 d^2 for every centroid within d of x
+            const double Au = (double)A * 1.0001;
+            const double bound = 2.0 * ((double)TcCfg<G>::ERR_UNITS * 5.9604644775390625e-8 *
+                                            (3.0 * Au + 4.0 * sqrt(Au * D) * 1.0000001 + 2.0 * D)
                                         + (double)invS * (6.103515625e-5 * (double)L1 * 1.0001 + norm_abs));
             if (!((double)keep_s2 - (double)keep_s1 > bound)) {
                 const ull slot = atomicAdd(reinterpret_cast<ull*>(status + 2), 1ull);

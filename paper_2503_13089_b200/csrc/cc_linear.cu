@@ -13,7 +13,9 @@
 //      item = 8 consecutive in_features x one code group (g consecutive out_features): 8 codes, 8
 //      codebook rows, transposed in registers into g rows of 16 bytes.
 //   B: NT tokens x 64 in_features of x (16-byte copies).
-// A ring of STAGES such stages feeds one MMA-issuing thread (4 MMAs of K = 16 per stage); full / empty
+// A ring of STAGES such stages feeds one MMA-issuing thread (4 MMAs of K = 16 per stage).  Each stage
+// belongs to its own four producer warps, so the gathers of four stages (codes, then codebook rows:
+// two dependent trips to L2) are in flight at once.  Full / empty
 // mbarriers, every wait bounded by a clock limit (a wait that runs out raises CC_DEV_TIMEOUT, the
 // CTA stops issuing work, skips its stores and still frees its tensor memory).
 // With few tokens and few 128-row tiles the in_features are split across CTAs (split-K): every split
@@ -29,7 +31,8 @@ namespace {
 constexpr int LM = 128;                 // out_features per CTA = MMA M = TMEM lanes
 constexpr int LKB = 64;                 // in_features per pipeline stage
 constexpr int LSTAGES = 4;
-constexpr int LPROD = 256;              // producer threads (8 warps); warps 0..3 also run the epilogue
+constexpr int LPROD = 512;              // producer threads (16 warps); warps 0..3 also run the epilogue
+constexpr int LSTAGE_THREADS = LPROD / LSTAGES;   // producer threads that fill one stage (four warps)
 constexpr int LTHREADS = LPROD + 32;    // + the MMA warp
 constexpr int LNT_MAX = 256;            // tokens per CTA = MMA N
 constexpr int A_STAGE = LM * LKB * 2;   // bytes
@@ -64,6 +67,28 @@ __device__ __forceinline__ void load_code_row(const uint16_t* __restrict__ C16, 
     }
 }
 
+// The same row as G / 2 32-bit words (even G).
+template <int G>
+__device__ __forceinline__ void load_code_row_words(const uint16_t* __restrict__ C16, int code, uint32_t* w) {
+    const uint16_t* row = C16 + (int64_t)code * G;
+    if constexpr (G % 8 == 0) {
+#pragma unroll
+        for (int v = 0; v < G / 8; ++v) {
+            const uint4 u = __ldg(reinterpret_cast<const uint4*>(row) + v);
+            w[4 * v] = u.x; w[4 * v + 1] = u.y; w[4 * v + 2] = u.z; w[4 * v + 3] = u.w;
+        }
+    } else if constexpr (G % 4 == 0) {
+#pragma unroll
+        for (int v = 0; v < G / 4; ++v) {
+            const uint2 u = __ldg(reinterpret_cast<const uint2*>(row) + v);
+            w[2 * v] = u.x; w[2 * v + 1] = u.y;
+        }
+    } else {
+#pragma unroll
+        for (int v = 0; v < G / 2; ++v) w[v] = __ldg(reinterpret_cast<const unsigned*>(row) + v);
+    }
+}
+
 // blockIdx.x: tile of 128 out_features; blockIdx.y: block of NT tokens; blockIdx.z: split of the
 // in_features (chunks_per_split stages each).  out: y itself (splits == 1) or this split's slab of
 // partial sums, both M x d_out FP32 row-major.
@@ -93,7 +118,7 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
 
     if (tid == 0) {
         for (int s = 0; s < LSTAGES; ++s) {
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(full + s)), "r"(LPROD));
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(full + s)), "r"(LSTAGE_THREADS));
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(empty + s)));
         }
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(acc_full)));
@@ -119,61 +144,103 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
         const int n_grp = grp_hi - grp_lo + 1;                      // >= 1: o0 < d_out <= out_groups * G
         const bool vec_x = (d_in % 8) == 0;
         bool ok = true;
-        for (int c = 0; c < n_chunks && ok; ++c) {
-            const int st = c % LSTAGES;
+        const int st = tid / LSTAGE_THREADS;                        // the stage this thread's group of warps fills
+        const int ptid = tid - st * LSTAGE_THREADS;
+        for (int c = st; c < n_chunks && ok; c += LSTAGES) {
             ok = mbar_wait(smem_u32(empty + st), ((c / LSTAGES) & 1) ^ 1, abort_flag);
             if (!ok) break;
             unsigned char* tA = sA + st * A_STAGE;
             unsigned char* tB = sB + st * b_stage;
             const int i0 = (chunk_first + c) * LKB;
             // ---- A: gather, transpose, store.  item = (block of 8 in_features, code group)
-            for (int item = tid; item < (LKB / 8) * n_grp; item += LPROD) {
+            for (int item = ptid; item < (LKB / 8) * n_grp; item += LSTAGE_THREADS) {
                 const int ib = item / n_grp, gl = item - ib * n_grp;
                 const int grp = grp_lo + gl;
-                uint16_t v[8][G];
+                if constexpr (G % 2 == 0) {
+                    // rows kept as 32-bit words (two out_features each): half the registers of a 16-bit copy
+                    uint32_t v[8][G / 2];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int i = i0 + ib * 8 + u;
-                    if (i < d_in) {
-                        const int code = __ldg(idx + (int64_t)i * out_groups + grp);
-                        load_code_row<G>(C16, code, v[u]);
-                    } else {
+                    for (int u = 0; u < 8; ++u) {
+                        const int i = i0 + ib * 8 + u;
+                        if (i < d_in) {
+                            const int code = __ldg(idx + (int64_t)i * out_groups + grp);
+                            load_code_row_words<G>(C16, code, v[u]);
+                        } else {
 #pragma unroll
-                        for (int t = 0; t < G; ++t) v[u][t] = 0;
+                            for (int t = 0; t < G / 2; ++t) v[u][t] = 0u;
+                        }
                     }
-                }
 #pragma unroll
-                for (int t = 0; t < G; ++t) {
-                    const int r = grp * G + t - o0;                 // row of the tile = out_feature - o0
-                    if (r < 0 || r >= LM) continue;
-                    uint4 w;
-                    w.x = (unsigned)v[0][t] | ((unsigned)v[1][t] << 16);
-                    w.y = (unsigned)v[2][t] | ((unsigned)v[3][t] << 16);
-                    w.z = (unsigned)v[4][t] | ((unsigned)v[5][t] << 16);
-                    w.w = (unsigned)v[6][t] | ((unsigned)v[7][t] << 16);
-                    *reinterpret_cast<uint4*>(tA + canon_bytes(r, ib * 8, LM)) = w;
+                    for (int t = 0; t < G; ++t) {
+                        const int r = grp * G + t - o0;             // row of the tile = out_feature - o0
+                        if (r < 0 || r >= LM) continue;
+                        const unsigned sel = (t & 1) ? 0x7632u : 0x5410u;   // high or low halves of two words
+                        uint4 w;
+                        w.x = __byte_perm(v[0][t / 2], v[1][t / 2], sel);
+                        w.y = __byte_perm(v[2][t / 2], v[3][t / 2], sel);
+                        w.z = __byte_perm(v[4][t / 2], v[5][t / 2], sel);
+                        w.w = __byte_perm(v[6][t / 2], v[7][t / 2], sel);
+                        *reinterpret_cast<uint4*>(tA + canon_bytes(r, ib * 8, LM)) = w;
+                    }
+                } else {
+                    uint16_t v[8][G];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        const int i = i0 + ib * 8 + u;
+                        if (i < d_in) {
+                            const int code = __ldg(idx + (int64_t)i * out_groups + grp);
+                            load_code_row<G>(C16, code, v[u]);
+                        } else {
+#pragma unroll
+                            for (int t = 0; t < G; ++t) v[u][t] = 0;
+                        }
+                    }
+#pragma unroll
+                    for (int t = 0; t < G; ++t) {
+                        const int r = grp * G + t - o0;
+                        if (r < 0 || r >= LM) continue;
+                        uint4 w;
+                        w.x = (unsigned)v[0][t] | ((unsigned)v[1][t] << 16);
+                        w.y = (unsigned)v[2][t] | ((unsigned)v[3][t] << 16);
+                        w.z = (unsigned)v[4][t] | ((unsigned)v[5][t] << 16);
+                        w.w = (unsigned)v[6][t] | ((unsigned)v[7][t] << 16);
+                        *reinterpret_cast<uint4*>(tA + canon_bytes(r, ib * 8, LM)) = w;
+                    }
                 }
             }
-            // ---- B: the tokens' slice of x, 8 in_features (16 bytes) at a time
-            for (int item = tid; item < NT * (LKB / 8); item += LPROD) {
-                const int kc = item % (LKB / 8), r = item / (LKB / 8);
-                const int m = m0 + r, i = i0 + kc * 8;
-                uint4 w = make_uint4(0u, 0u, 0u, 0u);
-                if (m < M && i < d_in) {
-                    const uint16_t* src = x + (int64_t)m * d_in + i;
-                    if (vec_x) {
-                        w = __ldg(reinterpret_cast<const uint4*>(src));
-                    } else {
-                        unsigned short h[8];
+            // ---- B: the tokens' slice of x, 8 in_features (16 bytes) at a time, four loads in flight per thread
+            const int n_b = NT * (LKB / 8);
+            for (int item0 = ptid; item0 < n_b; item0 += 4 * LSTAGE_THREADS) {
+                uint4 w[4];
 #pragma unroll
-                        for (int u = 0; u < 8; ++u) h[u] = (i + u < d_in) ? __ldg(src + u) : (unsigned short)0;
-                        w.x = (unsigned)h[0] | ((unsigned)h[1] << 16);
-                        w.y = (unsigned)h[2] | ((unsigned)h[3] << 16);
-                        w.z = (unsigned)h[4] | ((unsigned)h[5] << 16);
-                        w.w = (unsigned)h[6] | ((unsigned)h[7] << 16);
+                for (int u4 = 0; u4 < 4; ++u4) {
+                    const int item = item0 + u4 * LSTAGE_THREADS;
+                    const int kc = item % (LKB / 8), r = item / (LKB / 8);
+                    const int m = m0 + r, i = i0 + kc * 8;
+                    w[u4] = make_uint4(0u, 0u, 0u, 0u);
+                    if (item < n_b && m < M && i < d_in) {
+                        const uint16_t* src = x + (int64_t)m * d_in + i;
+                        if (vec_x) {
+                            w[u4] = __ldg(reinterpret_cast<const uint4*>(src));
+                        } else {
+                            unsigned short h[8];
+#pragma unroll
+                            for (int u = 0; u < 8; ++u) h[u] = (i + u < d_in) ? __ldg(src + u) : (unsigned short)0;
+                            w[u4].x = (unsigned)h[0] | ((unsigned)h[1] << 16);
+                            w[u4].y = (unsigned)h[2] | ((unsigned)h[3] << 16);
+                            w[u4].z = (unsigned)h[4] | ((unsigned)h[5] << 16);
+                            w[u4].w = (unsigned)h[6] | ((unsigned)h[7] << 16);
+                        }
                     }
                 }
-                *reinterpret_cast<uint4*>(tB + canon_bytes(r, kc * 8, NT)) = w;
+#pragma unroll
+                for (int u4 = 0; u4 < 4; ++u4) {
+                    const int item = item0 + u4 * LSTAGE_THREADS;
+                    if (item < n_b) {
+                        const int kc = item % (LKB / 8), r = item / (LKB / 8);
+                        *reinterpret_cast<uint4*>(tB + canon_bytes(r, kc * 8, NT)) = w[u4];
+                    }
+                }
             }
             asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // generic-proxy writes -> async proxy (MMA)
             asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(full + st)) : "memory");
@@ -263,7 +330,9 @@ LinearPlan linear_plan(int64_t M, int64_t d_out, int64_t d_in, int sm_count) {
     p.o_tiles = (int)((d_out + LM - 1) / LM);
     p.tok_blocks = (int)((M + p.NT - 1) / p.NT);
     const int chunks = (int)((d_in + LKB - 1) / LKB);
-    int splits = sm_count / (p.o_tiles * p.tok_blocks);             // fill the SMs when there are few tiles
+    // fill the SMs when there are few tiles; a narrow token block leaves room for several CTAs per SM, and the
+    // gathers are bound by latency, so more of them in flight is what helps
+    int splits = (p.NT <= 64 ? 4 * sm_count : sm_count) / (p.o_tiles * p.tok_blocks);
     if (splits > chunks / 4) splits = chunks / 4;                   // at least four stages of work per CTA
     if (splits < 1) splits = 1;
     p.chunks_per_split = (chunks + splits - 1) / splits;

@@ -74,7 +74,7 @@ def _gpu_update_rule(X, idx, C_prev, rule):
 
 
 @pytest.mark.parametrize("N,g,K,used", [(5000, 4, 64, 40), (70001, 4, 1000, 700), (100000, 6, 65536, 65536),
-                                        (3000, 16, 5000, 5000), (2000, 8, 300, 1), (500, 3, 40, 40)])
+                                        (3000, 16, 5000, 5000), (2000, 8, 300, 1), (500, 3, 40, 33)])
 def test_update_with_split_rule_matches_oracle_bit_for_bit(N, g, K, used):
     """M-step followed by the splitting rule; `used` codes are drawn from, the other clusters (and, with
     more clusters than points, many more) are empty.  With `used` = 1 one cluster donates again and again."""

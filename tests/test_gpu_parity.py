@@ -68,11 +68,12 @@ def test_decode_accepts_codes_that_are_only_two_byte_aligned():
     assert np.array_equal(u.u16_np(What.view(torch.uint16)).reshape(d_out, d_in), want.view(np.uint16))
 
 
-@pytest.mark.parametrize("g,K", [(4, 3000), (8, 2900), (16, 1400), (4, 1), (8, 6400), (16, 3000), (4, 65536)])
+@pytest.mark.parametrize("g,K", [(4, 3000), (8, 2900), (16, 1400), (4, 1), (8, 6400), (16, 3000), (4, 65536),
+                                 (8, 65536), (4, 40000), (8, 20001), (8, 9000), (16, 65536), (4, 16385)])
 def test_decode_of_a_large_matrix_matches_oracle(g, K):
     """Matrices with at least 8 tiles per SM: g = 8 and 16 with a codebook of at most 128 KB take the
-    persistent kernel (codebooks of at most 46 KB staged in shared memory), the others the plain
-    tiled kernel; ragged tiles on both edges."""
+    persistent kernel (codebooks of at most 46 KB staged in shared memory), the others -- among them
+    codebooks of 320 KB, 512 KB, 1 MB and 2 MB -- the plain tiled kernel.  Ragged tiles on both edges."""
     cc, u = _cc(), _u()
     d_out, d_in = 2056, 2568
     rng = np.random.default_rng(g * 100003 + K)
@@ -342,7 +343,11 @@ def test_assign_reports_nonfinite_input():
 # ------------------------------------------------------------------ M-step
 
 @pytest.mark.parametrize("N,g,K", [(1, 4, 3), (5000, 4, 64), (70001, 4, 1000), (9000, 8, 5000), (6000, 16, 129),
-                                   (3001, 5, 17), (3001, 9, 200), (4000, 1, 7)])
+                                   (3001, 5, 17), (3001, 9, 200), (4000, 1, 7),
+                                   # large inputs with accumulators that fit one SM: the shared-memory kernel
+                                   (400001, 4, 300), (1500000, 16, 1400), (2000000, 4, 4096), (900000, 7, 2000),
+                                   # ... and with accumulators that do not: L2 reductions
+                                   (3000003, 4, 65536), (2000000, 9, 65500)])
 def test_update_matches_oracle_bit_for_bit(N, g, K):
     u = _u()
     X = wl.make_points(N, g, 3000 + N)
@@ -357,10 +362,13 @@ def test_update_matches_oracle_bit_for_bit(N, g, K):
     assert np.array_equal(C_gpu[counts_or == 0].view(np.uint32), C_prev[counts_or == 0].view(np.uint32))
 
 
-def test_update_large_and_tiny_values_and_point_order():
+@pytest.mark.parametrize("N", [20000, 200000])
+def test_update_large_and_tiny_values_and_point_order(N):
+    """Values on the coarse accumulator (|x| >= 8), subnormals, a fixed point order and a shuffled one;
+    the larger size takes the shared-memory kernel."""
     u = _u()
     rng = np.random.default_rng(3)
-    X = wl.make_points(20000, 4, 77)
+    X = wl.make_points(N, 4, 77)
     X[::7] = (rng.standard_normal((len(X[::7]), 4)) * 300).astype(np.float16)       # |x| >= 8 accumulator
     X[::11] = (rng.standard_normal((len(X[::11]), 4)) * 1e-6).astype(np.float16)    # subnormals
     idx = rng.integers(0, 50, len(X)).astype(np.int32)
@@ -369,6 +377,7 @@ def test_update_large_and_tiny_values_and_point_order():
     C_gpu, counts_gpu = u.gpu_update(X, idx, C_prev)
     assert np.array_equal(counts_gpu, counts_or)
     assert u.centroid_rel_err(C_gpu, C_or, X) <= u.REL_CENTROID
+    assert np.array_equal(C_gpu.view(np.uint32), C_or.view(np.uint32))
     p = rng.permutation(len(X))
     C_perm, _ = u.gpu_update(X[p], idx[p], C_prev)
     assert np.array_equal(C_perm.view(np.uint32), C_gpu.view(np.uint32))

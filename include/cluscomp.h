@@ -101,8 +101,9 @@ int64_t cc_launch_count(const cc_ctx* ctx);
 #define CC_KERNEL_OTHER 8
 #define CC_KERNEL_ASSIGN_FINISH 9 /* tensor path: index, distance, near-tie flag per point */
 #define CC_KERNEL_UPDATE_DELTA 10  /* M-step inside cc_fit: only the points whose code changed */
-#define CC_KERNEL_LINEAR 11        /* forward of the compressed linear layer (GEMM + split reduction) */
-#define CC_KERNEL_CLASSES 12
+#define CC_KERNEL_LINEAR 11        /* forward of the compressed linear layer: the GEMM with the gathered weight */
+#define CC_KERNEL_LINEAR_REDUCE 12 /* ... and the sum of its split-K partial results                          */
+#define CC_KERNEL_CLASSES 13
 cc_status cc_profile_enable(cc_ctx* ctx, int on);
 cc_status cc_profile_read(cc_ctx* ctx, double* total_ms_host, int64_t* launches_host);
 

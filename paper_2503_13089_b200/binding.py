@@ -168,7 +168,7 @@ def cc_launch_count(ctx: Context) -> int:
 
 
 KERNEL_CLASSES = ("assign_main", "assign_prep", "resolve", "objective", "update_accum", "update_finish",
-                  "reshape", "decode", "other", "assign_finish", "update_delta", "linear")
+                  "reshape", "decode", "other", "assign_finish", "update_delta", "linear", "linear_reduce")
 
 
 def cc_profile_enable(ctx: Context, on: bool) -> None:

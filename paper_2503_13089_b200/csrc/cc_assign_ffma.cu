@@ -305,8 +305,39 @@ resolve_scan_kernel(const uint16_t* __restrict__ X, int64_t N, const float* __re
         }
         float bound = __double2float_ru(Db * (1.0 + 3.814697265625e-6));
         const int j_end = (sl + 1) * L < K ? (sl + 1) * L : K;
-#pragma unroll 2
-        for (int j = sl * L; j < j_end; ++j) {
+        // four centroids per round: their screening distances are independent chains, and only a round that
+        // holds a candidate looks closer
+        int j = sl * L;
+        for (; j + 4 <= j_end; j += 4) {
+            float dq[4];
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                float c[G];
+                load_centroid<G>(C, j + q, c);
+                dq[q] = 0.f;
+#pragma unroll
+                for (int t = 0; t < G; ++t) { const float df = x[t] - c[t]; dq[q] = fmaf(df, df, dq[q]); }
+            }
+            if (fminf(fminf(dq[0], dq[1]), fminf(dq[2], dq[3])) > bound) continue;
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                if (dq[q] <= bound) {
+                    float c[G];
+                    load_centroid<G>(C, j + q, c);
+                    double d = 0.0;
+#pragma unroll
+                    for (int t = 0; t < G; ++t) {
+                        const double df = __dsub_rn((double)x[t], (double)c[t]);
+                        d = __dadd_rn(d, __dmul_rn(df, df));
+                    }
+                    if (d < Db || (d == Db && j + q < jb)) {
+                        Db = d; jb = j + q;
+                        bound = __double2float_ru(Db * (1.0 + 3.814697265625e-6));
+                    }
+                }
+            }
+        }
+        for (; j < j_end; ++j) {
             float c[G];
             load_centroid<G>(C, j, c);
             float dh = 0.f;

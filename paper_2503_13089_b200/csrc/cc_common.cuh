@@ -14,7 +14,7 @@
 // Kernel classes for the optional per-kernel event timing (cc_profile_*).
 enum { CC_K_ASSIGN_MAIN = 0, CC_K_ASSIGN_PREP = 1, CC_K_RESOLVE = 2, CC_K_OBJECTIVE = 3, CC_K_UPDATE_ACCUM = 4,
        CC_K_UPDATE_FINISH = 5, CC_K_RESHAPE = 6, CC_K_DECODE = 7, CC_K_OTHER = 8, CC_K_ASSIGN_FINISH = 9, CC_K_UPDATE_DELTA = 10,
-       CC_K_LINEAR = 11, CC_K_COUNT = 12 };
+       CC_K_LINEAR = 11, CC_K_LINEAR_REDUCE = 12, CC_K_COUNT = 13 };
 constexpr int CC_PROF_CAP = 8192;
 
 struct cc_prof_slot { cudaEvent_t a, b; int kind; };

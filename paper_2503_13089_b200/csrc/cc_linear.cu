@@ -153,43 +153,68 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
             unsigned char* tB = sB + st * b_stage;
             const int i0 = (chunk_first + c) * LKB;
             // ---- A: gather, transpose, store.  item = (block of 8 in_features, code group)
-            for (int item = ptid; item < (LKB / 8) * n_grp; item += LSTAGE_THREADS) {
-                const int ib = item / n_grp, gl = item - ib * n_grp;
-                const int grp = grp_lo + gl;
+            // IPT items per thread and pass: all their codes are requested first, then all their rows, so that a
+            // pass costs two trips to L2 whatever IPT is (the rows of IPT items must fit the registers)
+            constexpr int IPT = (G % 2 == 0 && G <= 8) ? 2 : 1;
+            for (int item0 = ptid; item0 < (LKB / 8) * n_grp; item0 += IPT * LSTAGE_THREADS) {
                 if constexpr (G % 2 == 0) {
                     // rows kept as 32-bit words (two out_features each): half the registers of a 16-bit copy
-                    uint32_t v[8][G / 2];
+                    uint32_t v[IPT][8][G / 2];
+                    int code[IPT][8];
+                    int ibs[IPT], grps[IPT];
 #pragma unroll
-                    for (int u = 0; u < 8; ++u) {
-                        const int i = i0 + ib * 8 + u;
-                        if (i < d_in) {
-                            const int code = __ldg(idx + (int64_t)i * out_groups + grp);
-                            load_code_row_words<G>(C16, code, v[u]);
-                        } else {
+                    for (int q = 0; q < IPT; ++q) {
+                        const int item = item0 + q * LSTAGE_THREADS;
+                        const bool live = item < (LKB / 8) * n_grp;
+                        ibs[q] = live ? item / n_grp : 0;
+                        grps[q] = live ? grp_lo + (item - ibs[q] * n_grp) : -1;
 #pragma unroll
-                            for (int t = 0; t < G / 2; ++t) v[u][t] = 0u;
+                        for (int u = 0; u < 8; ++u) {
+                            const int i = i0 + ibs[q] * 8 + u;
+                            code[q][u] = (live && i < d_in) ? (int)__ldg(idx + (int64_t)i * out_groups + grps[q]) : -1;
                         }
                     }
 #pragma unroll
-                    for (int t = 0; t < G; ++t) {
-                        const int r = grp * G + t - o0;             // row of the tile = out_feature - o0
-                        if (r < 0 || r >= LM) continue;
-                        const unsigned sel = (t & 1) ? 0x7632u : 0x5410u;   // high or low halves of two words
-                        uint4 w;
-                        w.x = __byte_perm(v[0][t / 2], v[1][t / 2], sel);
-                        w.y = __byte_perm(v[2][t / 2], v[3][t / 2], sel);
-                        w.z = __byte_perm(v[4][t / 2], v[5][t / 2], sel);
-                        w.w = __byte_perm(v[6][t / 2], v[7][t / 2], sel);
-                        *reinterpret_cast<uint4*>(tA + canon_bytes(r, ib * 8, LM)) = w;
+                    for (int q = 0; q < IPT; ++q) {
+#pragma unroll
+                        for (int u = 0; u < 8; ++u) {
+                            if (code[q][u] >= 0) {
+                                load_code_row_words<G>(C16, code[q][u], v[q][u]);
+                            } else {
+#pragma unroll
+                                for (int t = 0; t < G / 2; ++t) v[q][u][t] = 0u;
+                            }
+                        }
+                    }
+#pragma unroll
+                    for (int q = 0; q < IPT; ++q) {
+                        if (grps[q] < 0) continue;
+#pragma unroll
+                        for (int t = 0; t < G; ++t) {
+                            const int r = grps[q] * G + t - o0;     // row of the tile = out_feature - o0
+                            if (r < 0 || r >= LM) continue;
+                            const unsigned sel = (t & 1) ? 0x7632u : 0x5410u;   // high or low halves of two words
+                            uint4 w;
+                            w.x = __byte_perm(v[q][0][t / 2], v[q][1][t / 2], sel);
+                            w.y = __byte_perm(v[q][2][t / 2], v[q][3][t / 2], sel);
+                            w.z = __byte_perm(v[q][4][t / 2], v[q][5][t / 2], sel);
+                            w.w = __byte_perm(v[q][6][t / 2], v[q][7][t / 2], sel);
+                            *reinterpret_cast<uint4*>(tA + canon_bytes(r, ibs[q] * 8, LM)) = w;
+                        }
                     }
                 } else {
+                    const int ib = item0 / n_grp, grp = grp_lo + (item0 - (item0 / n_grp) * n_grp);
                     uint16_t v[8][G];
+                    int code[8];
 #pragma unroll
                     for (int u = 0; u < 8; ++u) {
                         const int i = i0 + ib * 8 + u;
-                        if (i < d_in) {
-                            const int code = __ldg(idx + (int64_t)i * out_groups + grp);
-                            load_code_row<G>(C16, code, v[u]);
+                        code[u] = (i < d_in) ? (int)__ldg(idx + (int64_t)i * out_groups + grp) : -1;
+                    }
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) {
+                        if (code[u] >= 0) {
+                            load_code_row<G>(C16, code[u], v[u]);
                         } else {
 #pragma unroll
                             for (int t = 0; t < G; ++t) v[u][t] = 0;
@@ -330,9 +355,7 @@ LinearPlan linear_plan(int64_t M, int64_t d_out, int64_t d_in, int sm_count) {
     p.o_tiles = (int)((d_out + LM - 1) / LM);
     p.tok_blocks = (int)((M + p.NT - 1) / p.NT);
     const int chunks = (int)((d_in + LKB - 1) / LKB);
-    // fill the SMs when there are few tiles; a narrow token block leaves room for several CTAs per SM, and the
-    // gathers are bound by latency, so more of them in flight is what helps
-    int splits = (p.NT <= 64 ? 4 * sm_count : sm_count) / (p.o_tiles * p.tok_blocks);
+    int splits = sm_count / (p.o_tiles * p.tok_blocks);             // fill the SMs when there are few tiles
     if (splits > chunks / 4) splits = chunks / 4;                   // at least four stages of work per CTA
     if (splits < 1) splits = 1;
     p.chunks_per_split = (chunks + splits - 1) / splits;
@@ -365,13 +388,13 @@ template <int G>
 cudaError_t launch_linear(cc_ctx* ctx, const LinearPlan& p, const uint16_t* x, int M, const uint16_t* C16,
                           const uint16_t* idx, int d_out, int d_in, int out_groups, float* out, int64_t split_stride,
                           const float* bias, unsigned* status, cudaStream_t st) {
-    static size_t attr_dev[64] = {};
-    size_t& have = attr_dev[ctx->device & 63];
-    if (have < p.smem) {
+    static bool attr_dev[64] = {};
+    bool& have = attr_dev[ctx->device & 63];
+    if (!have) {
         const cudaError_t e = cudaFuncSetAttribute(linear_forward_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                    (int)(LSTAGES * (A_STAGE + LNT_MAX * LKB * 2) + 256));
         if (e != cudaSuccess) return e;
-        have = LSTAGES * (A_STAGE + LNT_MAX * LKB * 2) + 256;
+        have = true;
     }
     const dim3 grid(p.o_tiles, p.tok_blocks, p.splits);
     linear_forward_kernel<G><<<grid, LTHREADS, p.smem, st>>>(x, M, C16, idx, d_out, d_in, out_groups, p.NT, p.tmem_cols,
@@ -402,7 +425,7 @@ cudaError_t cc_launch_linear_forward(cc_ctx* ctx, const uint16_t* x, int64_t M, 
     }
     if (e != cudaSuccess) return e;
     if (p.splits > 1) {
-        ProfScope ps(ctx, CC_K_LINEAR, st);
+        ProfScope ps(ctx, CC_K_LINEAR_REDUCE, st);
         int64_t blocks = (n + 255) / 256;
         const int64_t cap = (int64_t)ctx->sm_count * 8;
         if (blocks > cap) blocks = cap;

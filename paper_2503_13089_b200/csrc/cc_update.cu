@@ -79,8 +79,10 @@ __global__ void __launch_bounds__(UP_THREADS, 1)
 update_private_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t* __restrict__ idx, int K,
                       ull* __restrict__ sum_lo, ull* __restrict__ sum_hi, int* __restrict__ counts) {
     extern __shared__ uint32_t up_sm[];
-    uint32_t* lo32 = up_sm;                          // K x G: low words of the biased sums
-    uint32_t* hi32 = lo32 + (size_t)K * G;           // K x G: carries
+    // coordinate-major (word t K + j): at step t a warp's 32 points hit banks j mod 32, spread over all
+    // banks, where the cluster-major order would confine them to the banks t mod G
+    uint32_t* lo32 = up_sm;                          // G x K: low words of the biased sums
+    uint32_t* hi32 = lo32 + (size_t)K * G;           // G x K: carries
     uint32_t* cnt = hi32 + (size_t)K * G;            // K
     for (int e = threadIdx.x; e < K * (2 * G + 1); e += UP_THREADS) up_sm[e] = 0u;
     __syncthreads();
@@ -103,16 +105,17 @@ update_private_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t*
             } else if (v == v) {
                 q += (uint32_t)__float2int_rn(v * 16777216.0f);      // |.| < 2^27
             }
-            const uint32_t old = atomicAdd(lo32 + j * G + t, q);
-            if (old + q < old) atomicAdd(hi32 + j * G + t, 1u);      // carry out of the low word
+            const uint32_t old = atomicAdd(lo32 + t * K + j, q);
+            if (old + q < old) atomicAdd(hi32 + t * K + j, 1u);      // carry out of the low word
         }
     }
     __syncthreads();
-    // add this block's sums to the global accumulators: one reduction per touched word
+    // add this block's sums to the global accumulators (cluster-major): one reduction per touched word
     for (int e = threadIdx.x; e < K * G; e += UP_THREADS) {
-        const uint32_t c = cnt[e / G];
+        const int j = e / G, t = e - j * G;
+        const uint32_t c = cnt[j];
         if (c == 0u) continue;
-        const ull v = (((ull)hi32[e] << 32) | (ull)lo32[e]) - ((ull)c << 27);
+        const ull v = (((ull)hi32[t * K + j] << 32) | (ull)lo32[t * K + j]) - ((ull)c << 27);
         if (v) atomicAdd(sum_lo + e, v);
     }
     for (int j = threadIdx.x; j < K; j += UP_THREADS)

@@ -27,11 +27,26 @@ def _worker(rank, world, port, out):
     os.environ["MASTER_ADDR"] = "127.0.0.1"
     os.environ["MASTER_PORT"] = str(port)
     dist.init_process_group("gloo", rank=rank, world_size=world)
+    import torch
+    from paper_2503_13089_b200 import binding as cc
     w = wl.WORKLOADS["cfg1_256x512_g4_k256"]
     specs = sharding.matrices_for_rank(w, rank)
     W = wl.make_matrix(specs[0])
     t = sharding.max_over_ranks(10.0 + rank)          # a stand-in for the rank's device time
-    out.put((rank, specs[0].data_seed, float(W.astype("float32").sum()), t))
+    # the benchmark's split of a job over the ranks: `world` copies of a 7B layer's matrices through the
+    # library's scheduler; the ranks exchange their shares and each checks that they partition the job
+    layer = wl.WORKLOADS["cfg5_layer7b_g16_k65536"]
+    job = [m for r in range(world) for m in sharding.matrices_for_rank(layer, r)]
+    sizes = [layer.n_subvectors(m) for m in job]
+    mine = cc.cc_schedule_matrices(sizes, world, rank)
+    flags = torch.zeros(len(job), dtype=torch.int64)
+    flags[mine] = 1
+    dist.all_reduce(flags)
+    load = torch.tensor([float(sum(sizes[i] for i in mine))], dtype=torch.float64)
+    loads = [torch.zeros(1, dtype=torch.float64) for _ in range(world)]
+    dist.all_gather(loads, load)
+    out.put((rank, specs[0].data_seed, float(W.astype("float32").sum()), t, bool((flags == 1).all()),
+             [float(v) for v in loads], float(sum(sizes))))
     dist.barrier()
     dist.destroy_process_group()
 
@@ -52,3 +67,7 @@ def test_two_gloo_ranks_take_different_matrices_and_share_max_time():
         assert p.exitcode == 0
     assert res[0][1] != res[1][1] and res[0][2] != res[1][2]      # different seeds, different data
     assert res[0][3] == res[1][3] == 11.0                          # both see the slower rank's time
+    assert res[0][4] and res[1][4]                                 # every matrix of the job went to exactly one rank
+    loads, total = res[0][5], res[0][6]
+    assert res[1][5] == loads and sum(loads) == total
+    assert max(loads) - min(loads) <= 2818048                      # balanced to within the largest matrix

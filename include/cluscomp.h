@@ -285,6 +285,10 @@ cc_status cc_set_empty_rule(cc_ctx* ctx, int rule);
  * final cc_assign over all N points against the fitted codebook fills idx / dist (N entries each; dist
  * may be NULL).  counts and objective_trace are those of the training set.  C: in = initial codebook. */
 int64_t cc_train_points(int64_t N, int K, int max_points_per_centroid);
+/* Host only: the first n entries of that seeded shuffle of 0..N-1 (0 <= n <= N < 2^31) as 32-bit
+ * positions -- the rows cc_fit_sampled trains on; for n <= 65536 the same positions as
+ * cc_init_positions. */
+cc_status cc_sample_positions(int64_t N, int64_t n, uint64_t seed, uint32_t* positions_host);
 cc_status cc_fit_sampled(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, int K, int iters, int max_points_per_centroid,
                          uint64_t seed, uint16_t* X_train, float* C, uint16_t* idx, float* dist, int32_t* counts,
                          double* objective_trace, void* stream);

@@ -60,6 +60,7 @@ SIGNATURES = {
     "cc_fit": (_i32, [_vp, _vp, _i64, _i32, _i32, _i32, _vp, _vp, _vp, _vp, _vp, _vp]),
     "cc_set_empty_rule": (_i32, [_vp, _i32]),
     "cc_train_points": (_i64, [_i64, _i32, _i32]),
+    "cc_sample_positions": (_i32, [_i64, _i64, _u64, _vp]),
     "cc_fit_sampled": (_i32, [_vp, _vp, _i64, _i32, _i32, _i32, _i32, _u64, _vp, _vp, _vp, _vp, _vp, _vp, _vp]),
     "cc_quantize_codebook": (_i32, [_vp, _vp, _i32, _i32, _i32, _vp, _vp, _vp, _vp]),
     "cc_schedule_matrices": (_i32, [_i32, _vp, _i32, _i32, _vp, _vp]),
@@ -293,6 +294,13 @@ def cc_set_empty_rule(ctx, rule: int) -> None:
 
 def cc_train_points(N: int, K: int, max_points_per_centroid: int) -> int:
     return int(load().cc_train_points(N, K, max_points_per_centroid))
+
+
+def cc_sample_positions(N: int, n: int, seed: int):
+    import numpy as np
+    pos = np.empty(max(n, 1), dtype=np.uint32)
+    _check(load().cc_sample_positions(N, n, seed, pos.ctypes.data_as(_vp)), "cc_sample_positions")
+    return pos[:n]
 
 
 def cc_fit_sampled(ctx, X, N, g, K, iters, max_points_per_centroid, seed, X_train, C, idx, dist, counts,

@@ -413,6 +413,12 @@ int64_t cc_train_points(int64_t N, int K, int max_points_per_centroid) {
     return n < N ? n : N;
 }
 
+cc_status cc_sample_positions(int64_t N, int64_t n, uint64_t seed, uint32_t* positions_host) {
+    if (!positions_host) return CC_ERR_NULL;
+    if (N < 1 || N >= (int64_t)1 << 31 || n < 0 || n > N) return CC_ERR_SHAPE;
+    return partial_shuffle_u32(N, n, seed, positions_host) ? CC_OK : CC_ERR_CUDA;
+}
+
 cc_status cc_fit_sampled(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, int K, int iters, int max_points_per_centroid,
                          uint64_t seed, uint16_t* X_train, float* C, uint16_t* idx, float* dist, int32_t* counts,
                          double* objective_trace, void* stream) {

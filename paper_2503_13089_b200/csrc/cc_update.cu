@@ -46,13 +46,26 @@ update_accumulate_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16
     sum_hi += (int64_t)copy * K * G;
     counts += (int64_t)copy * K;
     const int64_t total = N * G;
-    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (int64_t)gridDim.x * blockDim.x) {
-        const int64_t i = e / G;
-        const int t = (int)(e - i * G);
-        const int j = idx[i];
-        if (j >= K) continue;
-        if (t == 0) atomicAdd(counts + j, 1);
-        add_coord(__ldg(X + e), sum_lo + (int64_t)j * G + t, sum_hi + (int64_t)j * G + t);
+    const int64_t stride = (int64_t)gridDim.x * blockDim.x;
+    constexpr int EB = 4;                            // elements per thread and round: their loads are issued together
+    for (int64_t e0 = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e0 < total; e0 += EB * stride) {
+        int jj[EB];
+        uint16_t hh[EB];
+#pragma unroll
+        for (int p = 0; p < EB; ++p) {
+            const int64_t e = e0 + p * stride;
+            jj[p] = (e < total) ? (int)__ldg(idx + e / G) : K;
+            hh[p] = (e < total) ? __ldg(X + e) : (uint16_t)0;
+        }
+#pragma unroll
+        for (int p = 0; p < EB; ++p) {
+            const int64_t e = e0 + p * stride;
+            const int j = jj[p];
+            if (j >= K) continue;
+            const int t = (int)(e % G);
+            if (t == 0) atomicAdd(counts + j, 1);
+            add_coord(hh[p], sum_lo + (int64_t)j * G + t, sum_hi + (int64_t)j * G + t);
+        }
     }
 }
 
@@ -87,26 +100,35 @@ update_private_kernel(const uint16_t* __restrict__ X, int64_t N, const uint16_t*
     for (int e = threadIdx.x; e < K * (2 * G + 1); e += UP_THREADS) up_sm[e] = 0u;
     __syncthreads();
     const int64_t stride = (int64_t)gridDim.x * UP_THREADS;
-#pragma unroll 2
-    for (int64_t i = (int64_t)blockIdx.x * UP_THREADS + threadIdx.x; i < N; i += stride) {
-        const unsigned j = __ldg(idx + i);
-        float x[G];
-        bool nf = false;
-        load_point<G>(X, i, N, x, nf);
-        if (j >= (unsigned)K) continue;
-        atomicAdd(cnt + j, 1u);
+    constexpr int PB = (G <= 8) ? 4 : 2;             // points per thread and round: their loads are issued together
+    for (int64_t i0 = (int64_t)blockIdx.x * UP_THREADS + threadIdx.x; i0 < N; i0 += PB * stride) {
+        unsigned jj[PB];
+        float xx[PB][G];
 #pragma unroll
-        for (int t = 0; t < G; ++t) {
-            const float v = x[t];
-            uint32_t q = 1u << 27;                   // the bias alone: a skipped or coarse value adds nothing else
-            if (fabsf(v) >= 8.0f) {
-                if (fabsf(v) <= 65504.0f)            // finite: multiple of 2^-7, straight to the global accumulator
-                    atomicAdd(sum_hi + (int64_t)j * G + t, (ull)__float2ll_rn(v * 128.0f));
-            } else if (v == v) {
-                q += (uint32_t)__float2int_rn(v * 16777216.0f);      // |.| < 2^27
+        for (int p = 0; p < PB; ++p) {
+            const int64_t i = i0 + p * stride;
+            bool nf = false;
+            jj[p] = (i < N) ? (unsigned)__ldg(idx + i) : 0xffffffffu;
+            load_point<G>(X, i, N, xx[p], nf);
+        }
+#pragma unroll
+        for (int p = 0; p < PB; ++p) {
+            const unsigned j = jj[p];
+            if (j >= (unsigned)K) continue;
+            atomicAdd(cnt + j, 1u);
+#pragma unroll
+            for (int t = 0; t < G; ++t) {
+                const float v = xx[p][t];
+                uint32_t q = 1u << 27;               // the bias alone: a skipped or coarse value adds nothing else
+                if (fabsf(v) >= 8.0f) {
+                    if (fabsf(v) <= 65504.0f)        // finite: multiple of 2^-7, straight to the global accumulator
+                        atomicAdd(sum_hi + (int64_t)j * G + t, (ull)__float2ll_rn(v * 128.0f));
+                } else if (v == v) {
+                    q += (uint32_t)__float2int_rn(v * 16777216.0f);      // |.| < 2^27
+                }
+                const uint32_t old = atomicAdd(lo32 + t * K + j, q);
+                if (old + q < old) atomicAdd(hi32 + t * K + j, 1u);      // carry out of the low word
             }
-            const uint32_t old = atomicAdd(lo32 + t * K + j, q);
-            if (old + q < old) atomicAdd(hi32 + t * K + j, 1u);      // carry out of the low word
         }
     }
     __syncthreads();

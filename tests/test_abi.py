@@ -101,3 +101,17 @@ def test_schedule_matrices_is_the_size_balanced_split():
             assert sorted(i for part in got for i in part) == list(range(n))
     with pytest.raises(cc.CCError):
         cc.cc_schedule_matrices([1, 2], 2, 2)
+
+
+def test_sample_positions_match_the_oracle_shuffle_on_both_host_paths():
+    """The training-set positions of a subsampled fit: few positions keep only the touched entries of
+    the shuffle, many keep the whole array; both must be the oracle's full-array shuffle."""
+    for N, n, seed in [(60000, 3000, 17), (60000, 20000, 17), (60000, 60000, 5), (1000, 0, 1), (1, 1, 9),
+                       (3000000, 400000, 2), (3000000, 1000, 2)]:
+        got = cc.cc_sample_positions(N, n, seed)
+        want = oracle.init_positions(N, n, seed) if n else np.empty(0, np.int64)
+        assert np.array_equal(got.astype(np.int64), want)
+        assert len(set(got.tolist())) == n
+    assert np.array_equal(cc.cc_sample_positions(5000, 700, 42).astype(np.int64), cc.cc_init_positions(5000, 700, 42))
+    with pytest.raises(cc.CCError):
+        cc.cc_sample_positions(10, 11, 0)

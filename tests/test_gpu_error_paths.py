@@ -52,11 +52,21 @@ class Args:
         self.nres = torch.full((1,), -3, dtype=torch.int64, device="cuda")
         self.scores = torch.full((8, 256), -4.0, dtype=torch.float32, device="cuda")
         self.scan = torch.zeros((N, 2), dtype=torch.float32, device="cuda")
+        self.xin = torch.full((8, D_IN), 0.5, dtype=torch.float16, device="cuda")
+        self.ybuf = torch.full((8 * D_OUT + 8,), -6.0, dtype=torch.float32, device="cuda")
+        self.y = self.ybuf[:8 * D_OUT].view(8, D_OUT)
+        self.y_odd = self.ybuf[1:8 * D_OUT + 1].view(8, D_OUT)
+        self.q8 = torch.full((K * G,), 0x55, dtype=torch.uint8, device="cuda")
+        self.scale = torch.full((1,), -7.0, dtype=torch.float32, device="cuda")
+        self.c16out = torch.full((K, G), -8.0, dtype=torch.float16, device="cuda")
+        self.xtbuf = torch.full((N * G + 8,), -9.0, dtype=torch.float16, device="cuda")
+        self.xtrain = self.xtbuf[:N * G].view(N, G)
+        self.xtrain_odd = self.xtbuf[1:N * G + 1].view(N, G)
         self.snapshot = None
 
     def outputs(self):
         return [self.xbuf, self.cbuf, self.c16buf, self.wbuf, self.idx, self.dist, self.counts, self.obj, self.nres,
-                self.scores]
+                self.scores, self.ybuf, self.q8, self.scale, self.c16out, self.xtbuf]
 
     def take_snapshot(self):
         torch.cuda.synchronize()
@@ -95,13 +105,20 @@ def _calls(a, o):
                                               v("C16", a.C16), v("idx", a.idx), a.dist, a.obj),
         "cc_decode": lambda: cc.cc_decode(ctx, v("C16", a.C16), v("K", K), v("g", G), v("idx", a.idx), v("d_out", D_OUT),
                                           v("d_in", D_IN), v("layout", 0), v("W", a.W)),
+        "cc_linear_forward": lambda: cc.cc_linear_forward(ctx, v("x", a.xin), v("M", 8), v("C16", a.C16), v("K", K), v("g", G),
+                                                          v("idx", a.idx), v("d_out", D_OUT), v("d_in", D_IN), None, v("y", a.y)),
+        "cc_quantize_codebook": lambda: cc.cc_quantize_codebook(ctx, v("C16", a.C16), v("K", K), v("g", G), v("bits", 8),
+                                                                v("q", a.q8), v("scale", a.scale), a.c16out),
+        "cc_fit_sampled": lambda: cc.cc_fit_sampled(ctx, v("X", a.X), v("N", N), v("g", G), v("K", K), v("iters", 1),
+                                                    v("mppc", 10), 3, v("Xt", a.xtrain), v("C", a.C), v("idx", a.idx),
+                                                    a.dist, v("counts", a.counts), a.obj),
         "cc_update_static": lambda: cc.cc_update_static(0, v("X", a.X), v("N", N), v("g", G), v("idx", a.idx), v("K", K),
                                                         v("C", a.C), v("counts", a.counts)),
     }
 
 
 NEEDS_WS = ["cc_init_codebook", "cc_assign", "cc_tensor_scores", "cc_tensor_finish_only", "cc_last_flagged", "cc_update",
-            "cc_codebook_grad", "cc_fit", "cc_finalize"]
+            "cc_codebook_grad", "cc_fit", "cc_finalize", "cc_fit_sampled"]
 
 CASES = []
 for fn in ("cc_reshape_subvectors", "cc_init_codebook", "cc_assign", "cc_tensor_scores", "cc_tensor_finish_only",
@@ -149,6 +166,20 @@ CASES += [
     ("cc_init_codebook", {"N": K - 1}, N_LT_K), ("cc_init_codebook", {"N": 0}, SHAPE),
     # layout constants
     ("cc_reshape_subvectors", {"layout": 2}, LAYOUT), ("cc_decode", {"layout": -1}, LAYOUT),
+    # the rows beyond the clustering path
+    ("cc_linear_forward", {"g": 0}, BAD_G), ("cc_linear_forward", {"g": 17}, BAD_G), ("cc_linear_forward", {"K": 0}, BAD_K),
+    ("cc_linear_forward", {"K": 65537}, BAD_K), ("cc_linear_forward", {"x": None}, NULL), ("cc_linear_forward", {"C16": None}, NULL),
+    ("cc_linear_forward", {"idx": None}, NULL), ("cc_linear_forward", {"y": None}, NULL), ("cc_linear_forward", {"M": 0}, SHAPE),
+    ("cc_linear_forward", {"d_in": 0}, SHAPE), ("cc_linear_forward", {"M": 1 << 30}, SHAPE),
+    ("cc_linear_forward", {"C16": "C16_odd"}, ALIGN), ("cc_linear_forward", {"y": "y_odd"}, ALIGN),
+    ("cc_quantize_codebook", {"g": 0}, BAD_G), ("cc_quantize_codebook", {"K": 65537}, BAD_K),
+    ("cc_quantize_codebook", {"bits": 2}, SHAPE), ("cc_quantize_codebook", {"bits": 16}, SHAPE),
+    ("cc_quantize_codebook", {"C16": None}, NULL), ("cc_quantize_codebook", {"q": None}, NULL),
+    ("cc_quantize_codebook", {"scale": None}, NULL),
+    ("cc_fit_sampled", {"g": 17}, BAD_G), ("cc_fit_sampled", {"K": 0}, BAD_K), ("cc_fit_sampled", {"X": None}, NULL),
+    ("cc_fit_sampled", {"Xt": None}, NULL), ("cc_fit_sampled", {"C": None}, NULL), ("cc_fit_sampled", {"counts": None}, NULL),
+    ("cc_fit_sampled", {"mppc": 0}, SHAPE), ("cc_fit_sampled", {"iters": -1}, SHAPE), ("cc_fit_sampled", {"N": 0}, SHAPE),
+    ("cc_fit_sampled", {"X": "X_odd"}, ALIGN), ("cc_fit_sampled", {"Xt": "xtrain_odd"}, ALIGN),
 ]
 
 

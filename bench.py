@@ -373,24 +373,34 @@ def linear_rows(cc, torch, ctx, peaks):
     C16 = (torch.randn((K, g), device="cuda", generator=gen) * 0.02).to(torch.float16)
     idx = torch.randint(-32768, 32768, (N,), device="cuda", generator=gen, dtype=torch.int16).view(torch.uint16)   # all 65536 codes
     rows = []
+    ctx.ensure_workspace(N, g, K)
+    q4 = torch.empty((K * g + 1) // 2, dtype=torch.uint8, device="cuda")
+    scale4 = torch.empty(1, dtype=torch.float32, device="cuda")
+    cc.cc_quantize_codebook(ctx, C16, K, g, 4, q4, scale4, None)
     for M in (1, 16, 256, 4096):
         x = (torch.randn((M, d_in), device="cuda", generator=gen) * 0.5).to(torch.float16)
         y = torch.empty((M, d_out), dtype=torch.float32, device="cuda")
         ctx.ensure_workspace(N, g, K, at_least=cc.cc_linear_workspace_bytes(ctx, M, d_out, d_in))
-        for _ in range(3):
-            cc.cc_linear_forward(ctx, x, M, C16, K, g, idx, d_out, d_in, None, y)
         reps = 20
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        a.record(torch.cuda.current_stream())
-        for _ in range(reps):
-            cc.cc_linear_forward(ctx, x, M, C16, K, g, idx, d_out, d_in, None, y)
-        b.record(torch.cuda.current_stream())
-        torch.cuda.synchronize()
-        ms = a.elapsed_time(b) / reps
+
+        def timed(call):
+            for _ in range(3):
+                call()
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            a.record(torch.cuda.current_stream())
+            for _ in range(reps):
+                call()
+            b.record(torch.cuda.current_stream())
+            torch.cuda.synchronize()
+            return a.elapsed_time(b) / reps
+
+        ms = timed(lambda: cc.cc_linear_forward(ctx, x, M, C16, K, g, idx, d_out, d_in, None, y))
+        # the same layer with the codebook quantised to 4 bits and held in shared memory (Section 5.3)
+        ms_q4 = timed(lambda: cc.cc_linear_forward_q4(ctx, x, M, q4, scale4, K, g, idx, d_out, d_in, None, y))
         flops = 2.0 * M * d_in * d_out
         by = 2.0 * N + 2.0 * K * g + 2.0 * M * d_in + 4.0 * M * d_out          # codes, codebook, x, y
-        rows.append({"M": M, "d_out": d_out, "d_in": d_in, "g": g, "K": K, "ms": ms,
+        rows.append({"M": M, "d_out": d_out, "d_in": d_in, "g": g, "K": K, "ms": ms, "ms_codebook_4bit": ms_q4,
                      "tflops": flops / (ms * 1e-3) / 1e12, "tensor_frac_of_measured_bf16": flops / (ms * 1e-3) / 1e12 / peaks["bf16_tflops"],
                      "algorithmic_GBs": by / (ms * 1e-3) / 1e9, "frac_of_hbm": by / (ms * 1e-3) / 1e9 / peaks["hbm_gbs"],
                      "bytes_fused": by, "bytes_decode_then_gemm": by + 2 * 2.0 * d_in * d_out,
@@ -406,7 +416,7 @@ def run_kernel_mode(a):
     N, g, K = a.N, a.g, a.K
     ctx = cc.Context(0)
     d_out, d_in = g * 1024, N // 1024
-    ctx.ensure_workspace(N, g, K, at_least=cc.cc_linear_workspace_bytes(ctx, a.M, d_out, max(d_in, 1)) if a.kernel == "linear" else 0)
+    ctx.ensure_workspace(N, g, K, at_least=cc.cc_linear_workspace_bytes(ctx, a.M, d_out, max(d_in, 1)) if a.kernel in ("linear", "linear_q4") else 0)
     cc.cc_set_path(ctx, {"auto": 0, "ffma": 1, "tensor": 2}[a.path])
     Xn = wl.make_points(N, g, 1)
     X = torch.from_numpy(Xn.view(np.int16)).cuda().view(torch.float16)
@@ -418,14 +428,17 @@ def run_kernel_mode(a):
     obj = torch.zeros(1, dtype=torch.float64, device="cuda")
     nres = torch.zeros(1, dtype=torch.int64, device="cuda")
     C16 = torch.empty((K, g), dtype=torch.float16, device="cuda")
-    if a.kernel in ("decode", "reshape", "linear"):
+    if a.kernel in ("decode", "reshape", "linear", "linear_q4"):
         assert d_in * 1024 == N, "N must be a multiple of 1024 for the reshape / decode / linear cases"
     W = torch.empty((d_out, d_in), dtype=torch.float16, device="cuda")
     cc.cc_assign(ctx, X, N, g, C, K, idx, dist, obj, nres)      # warm-up; also valid codes for update / decode
     cc.cc_finalize(ctx, X, N, g, C, K, C16, idx, dist, obj)
     C2 = C.clone()
     X2 = torch.empty_like(X)
-    if a.kernel == "linear":
+    if a.kernel in ("linear", "linear_q4"):
+        q4 = torch.empty((K * g + 1) // 2, dtype=torch.uint8, device="cuda")
+        scale4 = torch.empty(1, dtype=torch.float32, device="cuda")
+        cc.cc_quantize_codebook(ctx, C16, K, g, 4, q4, scale4, None)
         xin = (torch.randn((a.M, d_in), device="cuda") * 0.5).to(torch.float16)
         y = torch.empty((a.M, d_out), dtype=torch.float32, device="cuda")
 
@@ -440,6 +453,8 @@ def run_kernel_mode(a):
             cc.cc_reshape_subvectors(ctx, W, d_out, d_in, g, cc.LAYOUT_PAPER_T, X2)
         elif a.kernel == "linear":
             cc.cc_linear_forward(ctx, xin, a.M, C16, K, g, idx, d_out, d_in, None, y)
+        elif a.kernel == "linear_q4":
+            cc.cc_linear_forward_q4(ctx, xin, a.M, q4, scale4, K, g, idx, d_out, d_in, None, y)
         else:
             cc.cc_fit(ctx, X, N, g, K, a.iters, C, idx, dist, counts, None)
 
@@ -467,7 +482,7 @@ def main():
     ap.add_argument("--path", default="auto", choices=["auto", "ffma", "tensor"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-secondary", action="store_true", help="skip the short runs of the other workloads")
-    ap.add_argument("--kernel", default=None, choices=["assign", "update", "decode", "reshape", "fit", "linear"])
+    ap.add_argument("--kernel", default=None, choices=["assign", "update", "decode", "reshape", "fit", "linear", "linear_q4"])
     ap.add_argument("--N", type=int, default=1 << 20)
     ap.add_argument("--g", type=int, default=4)
     ap.add_argument("--K", type=int, default=4096)

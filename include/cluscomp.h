@@ -350,6 +350,19 @@ cc_status cc_linear_forward(cc_ctx* ctx, const uint16_t* x, int64_t M, const uin
                             const uint16_t* idx, int64_t d_out, int64_t d_in, const float* bias, float* y,
                             void* stream);
 
+/* The same forward with the codebook quantised to 4 bits (Section 5.3, "Inference latency": for
+ * inference the codebook may be quantised uniformly, and it is the 4-bit codebook that speeds the layer
+ * up).  q and scale are what cc_quantize_codebook(bits = 4) wrote: ceil(K * g / 2) bytes, element 2k in
+ * the low nibble, and one device float.  The weight is the dequantised codebook, value = round-to-nearest-
+ * even FP16 of nibble * scale -- exactly the C16_dequantized of cc_quantize_codebook, so the result equals
+ * cc_linear_forward on that codebook.  The packed codebook (at most 128 KB: K * g <= 262144) is held in
+ * every thread block's shared memory, which turns the gathers from requests to L2 into shared-memory
+ * reads.  g even (2..16; other g: CC_ERR_UNSUPPORTED_G); a larger codebook: CC_ERR_SHAPE; q 16-byte
+ * aligned; workspace as for cc_linear_forward. */
+cc_status cc_linear_forward_q4(cc_ctx* ctx, const uint16_t* x, int64_t M, const uint8_t* q, const float* scale, int K,
+                               int g, const uint16_t* idx, int64_t d_out, int64_t d_in, const float* bias, float* y,
+                               void* stream);
+
 /* Waits for `stream`, reads the device status word and clears it.  Returns CC_OK,
  * CC_ERR_NONFINITE, CC_ERR_DEVICE_TIMEOUT or CC_ERR_CUDA. */
 cc_status cc_poll_status(cc_ctx* ctx, void* stream);

@@ -69,6 +69,7 @@ SIGNATURES = {
     "cc_decode": (_i32, [_vp, _vp, _i32, _i32, _vp, _i64, _i64, _i32, _vp, _vp]),
     "cc_linear_workspace_bytes": (_sz, [_vp, _i64, _i64, _i64]),
     "cc_linear_forward": (_i32, [_vp, _vp, _i64, _vp, _i32, _i32, _vp, _i64, _i64, _vp, _vp, _vp]),
+    "cc_linear_forward_q4": (_i32, [_vp, _vp, _i64, _vp, _vp, _i32, _i32, _vp, _i64, _i64, _vp, _vp, _vp]),
     "cc_poll_status": (_i32, [_vp, _vp]),
     "cc_compress_host": (_i32, [_vp, _vp, _i64, _i64, _i32, _i32, _i32, _u64, _i32, _vp, _vp, _vp, _vp, _vp]),
 }
@@ -358,6 +359,11 @@ def cc_linear_workspace_bytes(ctx, M: int, d_out: int, d_in: int) -> int:
 def cc_linear_forward(ctx, x, M, C16, K, g, idx, d_out, d_in, bias, y, stream=None) -> None:
     _check(load().cc_linear_forward(ctx._h, _ptr(x), M, _ptr(C16), K, g, _ptr(idx), d_out, d_in, _ptr(bias), _ptr(y),
                                     _stream(stream)), "cc_linear_forward")
+
+
+def cc_linear_forward_q4(ctx, x, M, q, scale, K, g, idx, d_out, d_in, bias, y, stream=None) -> None:
+    _check(load().cc_linear_forward_q4(ctx._h, _ptr(x), M, _ptr(q), _ptr(scale), K, g, _ptr(idx), d_out, d_in, _ptr(bias),
+                                       _ptr(y), _stream(stream)), "cc_linear_forward_q4")
 
 
 def cc_poll_status(ctx, stream=None) -> None:

@@ -550,7 +550,23 @@ cc_status cc_linear_forward(cc_ctx* ctx, const uint16_t* x, int64_t M, const uin
     if (!aligned16(x) || !aligned16(C16) || !aligned16(y)) return CC_ERR_ALIGN;
     if (!ctx->ws || ctx->ws_bytes < cc_linear_scratch_bytes(M, d_out, d_in, ctx->sm_count)) return CC_ERR_WORKSPACE;
     if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
-    return from_cuda(cc_launch_linear_forward(ctx, x, M, C16, K, g, idx, d_out, d_in, bias, y, (cudaStream_t)stream));
+    return from_cuda(cc_launch_linear_forward(ctx, x, M, C16, nullptr, nullptr, K, g, idx, d_out, d_in, bias, y,
+                                              (cudaStream_t)stream));
+}
+
+cc_status cc_linear_forward_q4(cc_ctx* ctx, const uint16_t* x, int64_t M, const uint8_t* q, const float* scale, int K, int g,
+                               const uint16_t* idx, int64_t d_out, int64_t d_in, const float* bias, float* y, void* stream) {
+    if (!ctx || !x || !q || !scale || !idx || !y) return CC_ERR_NULL;
+    if (g < 2 || g > 16 || (g & 1)) return CC_ERR_UNSUPPORTED_G;
+    if (K < 1 || K > 65536) return CC_ERR_K_RANGE;
+    const int64_t N = cc_num_subvectors(d_out, d_in, g, CC_LAYOUT_PAPER_T);
+    if (N < 1 || N >= (int64_t)1 << 31 || M < 1 || M * d_out >= (int64_t)1 << 31) return CC_ERR_SHAPE;
+    if ((int64_t)K * (g / 2) > cc_linear_q_table_max()) return CC_ERR_SHAPE;
+    if (!aligned16(x) || !aligned16(q) || !aligned16(y)) return CC_ERR_ALIGN;
+    if (!ctx->ws || ctx->ws_bytes < cc_linear_scratch_bytes(M, d_out, d_in, ctx->sm_count)) return CC_ERR_WORKSPACE;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
+    return from_cuda(cc_launch_linear_forward(ctx, x, M, nullptr, q, scale, K, g, idx, d_out, d_in, bias, y,
+                                              (cudaStream_t)stream));
 }
 
 cc_status cc_poll_status(cc_ctx* ctx, void* stream) {

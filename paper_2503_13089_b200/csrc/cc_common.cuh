@@ -122,9 +122,10 @@ cudaError_t cc_launch_assign_tail(cc_ctx*, const WsLayout&, const uint16_t* X, i
 
 // Compressed linear layer: y = x . decode(C16, idx)^T (+ bias), the decoded weight never stored.
 size_t cc_linear_scratch_bytes(int64_t M, int64_t d_out, int64_t d_in, int sm_count);
-cudaError_t cc_launch_linear_forward(cc_ctx*, const uint16_t* x, int64_t M, const uint16_t* C16, int K, int g,
-                                     const uint16_t* idx, int64_t d_out, int64_t d_in, const float* bias, float* y,
-                                     cudaStream_t);
+int cc_linear_q_table_max(void);
+cudaError_t cc_launch_linear_forward(cc_ctx*, const uint16_t* x, int64_t M, const uint16_t* C16, const unsigned char* qtab,
+                                     const float* qscale, int K, int g, const uint16_t* idx, int64_t d_out, int64_t d_in,
+                                     const float* bias, float* y, cudaStream_t);
 
 cudaError_t cc_launch_quantize_codebook(cc_ctx*, const uint16_t* C16, int64_t n, int bits, uint8_t* q, float* scale,
                                         uint16_t* deq, cudaStream_t);

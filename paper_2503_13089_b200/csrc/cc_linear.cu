@@ -89,12 +89,28 @@ __device__ __forceinline__ void load_code_row_words(const uint16_t* __restrict__
     }
 }
 
+// Quantised codebook (4 bits per value, two values per byte, low nibble first; Section 5.3): the whole
+// table sits in shared memory, and a 256-entry table turns a byte into its two dequantised FP16 values
+// (value = round-to-nearest-even FP16 of nibble * scale, the nibble a two's-complement number).
+constexpr int LQ_TABLE_MAX = 128 * 1024;   // bytes of packed codebook that fit beside the stages
+constexpr int LQ_NT_MAX = 64;              // tokens per CTA when the table takes most of the shared memory
+
+template <int G>
+__device__ __forceinline__ void load_code_row_words_q(const unsigned char* __restrict__ qt,
+                                                      const uint32_t* __restrict__ lut2, int code, uint32_t* w) {
+    const unsigned char* row = qt + code * (G / 2);
+#pragma unroll
+    for (int v = 0; v < G / 2; ++v) w[v] = lut2[row[v]];
+}
+
 // blockIdx.x: tile of 128 out_features; blockIdx.y: block of NT tokens; blockIdx.z: split of the
 // in_features (chunks_per_split stages each).  out: y itself (splits == 1) or this split's slab of
 // partial sums, both M x d_out FP32 row-major.
-template <int G>
+// QUANT: the codebook is the packed 4-bit table `qtab` (K G / 2 bytes) with its scale instead of C16.
+template <int G, bool QUANT>
 __global__ void __launch_bounds__(LTHREADS, 1)
 linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __restrict__ C16,
+                      const unsigned char* __restrict__ qtab, const float* __restrict__ qscale, int K,
                       const uint16_t* __restrict__ idx, int d_out, int d_in, int out_groups, int NT,
                       int tmem_cols, int chunks_per_split, float* __restrict__ out, int64_t split_stride,
                       const float* __restrict__ bias, unsigned* __restrict__ status) {
@@ -106,6 +122,8 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
     uint64_t* full = bars, *empty = bars + LSTAGES, *acc_full = bars + 2 * LSTAGES;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * LSTAGES + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    uint32_t* lut2 = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(bars) + 256);   // QUANT only
+    unsigned char* qt = reinterpret_cast<unsigned char*>(lut2 + 256);                            // QUANT only
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int o0 = blockIdx.x * LM;
@@ -129,6 +147,20 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
                      "r"(tmem_cols));
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    if constexpr (QUANT) {
+        // the packed codebook and the byte -> two FP16 values table, once per CTA
+        const float s = __ldg(qscale);
+        if (tid < 256) {
+            const int lo = ((tid & 15) ^ 8) - 8, hi = ((tid >> 4) ^ 8) - 8;     // sign-extended nibbles
+            const unsigned a = __half_as_ushort(__float2half_rn(__fmul_rn((float)lo, s)));
+            const unsigned b = __half_as_ushort(__float2half_rn(__fmul_rn((float)hi, s)));
+            lut2[tid] = a | (b << 16);
+        }
+        const int bytes = K * (G / 2);
+        for (int v = tid; v < bytes / 16; v += LTHREADS)
+            reinterpret_cast<uint4*>(qt)[v] = __ldg(reinterpret_cast<const uint4*>(qtab) + v);
+        for (int v = (bytes / 16) * 16 + tid; v < bytes; v += LTHREADS) qt[v] = __ldg(qtab + v);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
@@ -179,7 +211,8 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
 #pragma unroll
                         for (int u = 0; u < 8; ++u) {
                             if (code[q][u] >= 0) {
-                                load_code_row_words<G>(C16, code[q][u], v[q][u]);
+                                if constexpr (QUANT) load_code_row_words_q<G>(qt, lut2, code[q][u], v[q][u]);
+                                else load_code_row_words<G>(C16, code[q][u], v[q][u]);
                             } else {
 #pragma unroll
                                 for (int t = 0; t < G / 2; ++t) v[q][u][t] = 0u;
@@ -346,9 +379,10 @@ linear_reduce_kernel(const float* __restrict__ partial, int splits, int64_t n, i
 
 struct LinearPlan { int NT, tmem_cols, o_tiles, tok_blocks, splits, chunks_per_split; size_t smem; };
 
-LinearPlan linear_plan(int64_t M, int64_t d_out, int64_t d_in, int sm_count) {
+// nt_max: tokens per CTA (256, or 64 with a quantised codebook in shared memory); table_bytes: that codebook.
+LinearPlan linear_plan(int64_t M, int64_t d_out, int64_t d_in, int sm_count, int nt_max = LNT_MAX, size_t table_bytes = 0) {
     LinearPlan p;
-    const int64_t mt = M < LNT_MAX ? M : LNT_MAX;
+    const int64_t mt = M < nt_max ? M : nt_max;
     p.NT = (int)((mt + 15) / 16 * 16);
     p.tmem_cols = 32;
     while (p.tmem_cols < p.NT) p.tmem_cols *= 2;
@@ -361,15 +395,21 @@ LinearPlan linear_plan(int64_t M, int64_t d_out, int64_t d_in, int sm_count) {
     p.chunks_per_split = (chunks + splits - 1) / splits;
     p.splits = (chunks + p.chunks_per_split - 1) / p.chunks_per_split;
     p.smem = (size_t)LSTAGES * (A_STAGE + (size_t)p.NT * LKB * 2) + 256;
+    if (table_bytes) p.smem += 1024 + (table_bytes + 15) / 16 * 16;
     return p;
 }
 
 }  // namespace
 
 size_t cc_linear_scratch_bytes(int64_t M, int64_t d_out, int64_t d_in, int sm_count) {
+    // enough for either form of the codebook: the quantised one takes narrower token blocks and may split more
     const LinearPlan p = linear_plan(M, d_out, d_in, sm_count);
-    return 256 + (p.splits > 1 ? (size_t)p.splits * (size_t)M * (size_t)d_out * 4 : 0);
+    const LinearPlan q = linear_plan(M, d_out, d_in, sm_count, LQ_NT_MAX, 16);
+    const int splits = p.splits > q.splits ? p.splits : q.splits;
+    return 256 + (splits > 1 ? (size_t)splits * (size_t)M * (size_t)d_out * 4 : 0);
 }
+
+int cc_linear_q_table_max(void) { return LQ_TABLE_MAX; }
 
 #define CC_LINEAR_DISPATCH(g, CALL)                                                                 \
     switch (g) {                                                                                    \
@@ -384,31 +424,36 @@ size_t cc_linear_scratch_bytes(int64_t M, int64_t d_out, int64_t d_in, int sm_co
 
 namespace {
 
-template <int G>
+template <int G, bool QUANT>
 cudaError_t launch_linear(cc_ctx* ctx, const LinearPlan& p, const uint16_t* x, int M, const uint16_t* C16,
-                          const uint16_t* idx, int d_out, int d_in, int out_groups, float* out, int64_t split_stride,
-                          const float* bias, unsigned* status, cudaStream_t st) {
+                          const unsigned char* qtab, const float* qscale, int K, const uint16_t* idx, int d_out, int d_in,
+                          int out_groups, float* out, int64_t split_stride, const float* bias, unsigned* status,
+                          cudaStream_t st) {
     static bool attr_dev[64] = {};
     bool& have = attr_dev[ctx->device & 63];
     if (!have) {
-        const cudaError_t e = cudaFuncSetAttribute(linear_forward_kernel<G>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   (int)(LSTAGES * (A_STAGE + LNT_MAX * LKB * 2) + 256));
+        const int max_smem = QUANT ? (int)(LSTAGES * (A_STAGE + LQ_NT_MAX * LKB * 2) + 256 + 1024 + LQ_TABLE_MAX)
+                                   : (int)(LSTAGES * (A_STAGE + LNT_MAX * LKB * 2) + 256);
+        const cudaError_t e = cudaFuncSetAttribute(linear_forward_kernel<G, QUANT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   max_smem);
         if (e != cudaSuccess) return e;
         have = true;
     }
     const dim3 grid(p.o_tiles, p.tok_blocks, p.splits);
-    linear_forward_kernel<G><<<grid, LTHREADS, p.smem, st>>>(x, M, C16, idx, d_out, d_in, out_groups, p.NT, p.tmem_cols,
-                                                             p.chunks_per_split, out, split_stride, bias, status);
+    linear_forward_kernel<G, QUANT><<<grid, LTHREADS, p.smem, st>>>(x, M, C16, qtab, qscale, K, idx, d_out, d_in, out_groups,
+                                                                    p.NT, p.tmem_cols, p.chunks_per_split, out, split_stride,
+                                                                    bias, status);
     return cudaGetLastError();
 }
 
 }  // namespace
 
-cudaError_t cc_launch_linear_forward(cc_ctx* ctx, const uint16_t* x, int64_t M, const uint16_t* C16, int K, int g,
-                                     const uint16_t* idx, int64_t d_out, int64_t d_in, const float* bias, float* y,
-                                     cudaStream_t st) {
-    (void)K;
-    const LinearPlan p = linear_plan(M, d_out, d_in, ctx->sm_count);
+// qtab == nullptr: FP16 codebook C16; otherwise the packed 4-bit codebook with its scale (even g only).
+cudaError_t cc_launch_linear_forward(cc_ctx* ctx, const uint16_t* x, int64_t M, const uint16_t* C16,
+                                     const unsigned char* qtab, const float* qscale, int K, int g, const uint16_t* idx,
+                                     int64_t d_out, int64_t d_in, const float* bias, float* y, cudaStream_t st) {
+    const LinearPlan p = qtab ? linear_plan(M, d_out, d_in, ctx->sm_count, LQ_NT_MAX, (size_t)K * (g / 2))
+                              : linear_plan(M, d_out, d_in, ctx->sm_count);
     char* ws = static_cast<char*>(ctx->ws);
     unsigned* status = reinterpret_cast<unsigned*>(ws);
     float* partial = reinterpret_cast<float*>(ws + 256);
@@ -419,9 +464,19 @@ cudaError_t cc_launch_linear_forward(cc_ctx* ctx, const uint16_t* x, int64_t M, 
         ProfScope ps(ctx, CC_K_LINEAR, st);
         float* out = p.splits > 1 ? partial : y;
         const float* b = p.splits > 1 ? nullptr : bias;
-#define CALL(G) e = launch_linear<G>(ctx, p, x, (int)M, C16, idx, (int)d_out, (int)d_in, out_groups, out, n, b, status, st)
-        CC_LINEAR_DISPATCH(g, CALL)
+        if (qtab) {
+#define CALL(G) e = launch_linear<G, true>(ctx, p, x, (int)M, nullptr, qtab, qscale, K, idx, (int)d_out, (int)d_in, out_groups, out, n, b, status, st)
+            switch (g) {
+                case 2: CALL(2); break;   case 4: CALL(4); break;   case 6: CALL(6); break;   case 8: CALL(8); break;
+                case 10: CALL(10); break; case 12: CALL(12); break; case 14: CALL(14); break; case 16: CALL(16); break;
+                default: return cudaErrorInvalidValue;
+            }
 #undef CALL
+        } else {
+#define CALL(G) e = launch_linear<G, false>(ctx, p, x, (int)M, C16, nullptr, nullptr, K, idx, (int)d_out, (int)d_in, out_groups, out, n, b, status, st)
+            CC_LINEAR_DISPATCH(g, CALL)
+#undef CALL
+        }
     }
     if (e != cudaSuccess) return e;
     if (p.splits > 1) {

@@ -92,3 +92,66 @@ def test_linear_forward_equals_decode_then_matmul():
     cc.cc_decode(u.ctx(), u.half_dev(C16), K, g, u.dev(idx.view(np.int16)).view(torch.uint16), d_out, d_in, 0, What)
     W_hat = What.cpu().numpy().astype(np.float64)
     _check(y, x.astype(np.float64) @ W_hat.T)
+
+
+# ------------------------------------------------------------------ 4-bit codebook (Section 5.3)
+
+def _gpu_forward_q4(x, C16, idx, d_out, d_in, bias):
+    """cc_quantize_codebook(bits = 4) on the device, then the forward on the packed codebook; also returns the
+    dequantised FP16 codebook the quantiser wrote."""
+    from paper_2503_13089_b200 import binding as cc
+    from tests import gpu_util as u
+    M = x.shape[0]
+    K, g = C16.shape
+    c = u.ctx()
+    c.ensure_workspace(len(idx), g, K, at_least=cc.cc_linear_workspace_bytes(c, M, d_out, d_in))
+    q = torch.zeros((K * g + 1) // 2, dtype=torch.uint8, device="cuda")
+    scale = torch.zeros(1, dtype=torch.float32, device="cuda")
+    deq = torch.zeros((K, g), dtype=torch.float16, device="cuda")
+    cc.cc_quantize_codebook(c, u.half_dev(C16), K, g, 4, q, scale, deq)
+    y = torch.full((M, d_out), float("nan"), dtype=torch.float32, device="cuda")
+    cc.cc_linear_forward_q4(c, u.half_dev(x), M, q, scale, K, g, u.dev(idx.view(np.int16)).view(torch.uint16), d_out, d_in,
+                            None if bias is None else u.dev(bias), y)
+    cc.cc_poll_status(c)
+    return y.cpu().numpy(), deq.cpu().numpy()
+
+
+@pytest.mark.parametrize("M,d_out,d_in,g,K", [
+    (1, 256, 512, 4, 256), (16, 1000, 520, 4, 700), (5, 130, 72, 6, 50), (9, 96, 72, 2, 40), (130, 144, 328, 12, 77),
+    (40, 512, 256, 8, 30000),       # 120,000 bytes of packed codebook
+    (24, 256, 128, 16, 16384),      # exactly the 131,072 bytes that fit
+    (33, 208, 136, 10, 21), (18, 300, 96, 14, 19),
+    (64, 4096, 4096, 4, 65536),     # the paper's largest codebook at g = 4: 128 KB packed
+    (200, 384, 256, 4, 65535),      # four token blocks of 64; an odd number of bytes
+])
+def test_linear_forward_q4_matches_oracle(M, d_out, d_in, g, K):
+    from paper_2503_13089_b200 import binding as cc
+    x, C16, idx, bias = _case(M, d_out, d_in, g, K, 3 * M + d_out + g)
+    q_or, s_or, deq_or = oracle.quantize_codebook(C16, 4)
+    y, deq_gpu = _gpu_forward_q4(x, C16, idx, d_out, d_in, bias)
+    assert np.array_equal(deq_gpu.view(np.uint16), deq_or.view(np.uint16))
+    want = oracle.linear_forward(x, deq_or, idx.astype(np.int32), d_out, d_in, bias)      # the layer on the dequantised codebook
+    _check(y, want)
+    y_fp16 = _gpu_forward(x, deq_or, idx, d_out, d_in, bias)                             # the FP16 kernel on the same codebook
+    if M <= 64:            # same token blocks and splits: the same sums in the same order
+        assert np.array_equal(y.view(np.uint32), y_fp16.view(np.uint32))
+    else:
+        _check(y_fp16, want)
+
+
+def test_linear_forward_q4_rejects_what_it_cannot_hold():
+    from paper_2503_13089_b200 import binding as cc
+    from tests import gpu_util as u
+    c = u.ctx()
+    c.ensure_workspace(70000, 4, 64)
+    x = torch.zeros((4, 64), dtype=torch.float16, device="cuda")
+    y = torch.full((4, 64), 5.0, dtype=torch.float32, device="cuda")
+    q = torch.zeros(1 << 20, dtype=torch.uint8, device="cuda")
+    scale = torch.ones(1, dtype=torch.float32, device="cuda")
+    idx = torch.zeros(64 * 64, dtype=torch.uint16, device="cuda")
+    for g, K, status in ((5, 64, 3), (1, 64, 3), (8, 65536, 2), (16, 16385, 2), (4, 0, 4)):
+        with pytest.raises(cc.CCError) as e:
+            cc.cc_linear_forward_q4(c, x, 4, q, scale, K, g, idx, 64, 64, None, y)
+        assert e.value.status == status, (g, K)
+    torch.cuda.synchronize()
+    assert bool((y == 5).all())

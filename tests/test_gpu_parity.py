@@ -86,6 +86,28 @@ def test_decode_of_a_large_matrix_matches_oracle(g, K):
     assert np.array_equal(u.u16_np(What.view(torch.uint16)).reshape(d_out, d_in), want.view(np.uint16))
 
 
+@pytest.mark.parametrize("g,d_out,K", [
+    (4, 2078, 1), (4, 2078, 3000), (4, 2078, 16385), (4, 2078, 19841), (4, 2078, 40000), (4, 2078, 65536),
+    (8, 2107, 2900), (8, 2107, 9000), (8, 2107, 10945), (8, 2107, 20001), (8, 2107, 65536),
+    (16, 2170, 1400), (16, 2170, 5000), (16, 2170, 5729), (16, 2170, 65536),
+])
+def test_decode_with_whole_sixteen_byte_code_rows_matches_oracle(g, d_out, K):
+    """Padded out_features a multiple of 8 g (every in_feature's code row is a whole number of 16-byte
+    pieces), codebooks from one row to 2 MB with every row used, ragged tiles on both edges, padded
+    out_features dropped."""
+    cc, u = _cc(), _u()
+    d_in = 2568
+    rng = np.random.default_rng(g * 7919 + K)
+    N = cc.cc_num_subvectors(d_out, d_in, g, 0)
+    C16 = rng.standard_normal((K, g)).astype(np.float16)
+    idx = rng.integers(0, K, N).astype(np.uint16)
+    idx[:K] = np.arange(K)[::-1].astype(np.uint16)     # every row is used
+    What = torch.zeros((d_out, d_in), dtype=torch.float16, device="cuda")
+    cc.cc_decode(u.ctx(), u.half_dev(C16), K, g, u.dev(idx.view(np.int16)).view(torch.uint16), d_out, d_in, 0, What)
+    want = oracle.decode(C16, idx.astype(np.int32), d_out, d_in, 0)
+    assert np.array_equal(u.u16_np(What.view(torch.uint16)).reshape(d_out, d_in), want.view(np.uint16))
+
+
 @pytest.mark.parametrize("N,g,K,seed", [(5000, 4, 700, 42), (257, 3, 257, 9), (100000, 8, 4096, 1)])
 def test_init_codebook_matches_oracle(N, g, K, seed):
     cc, u = _cc(), _u()

@@ -354,11 +354,15 @@ cc_status cc_linear_forward(cc_ctx* ctx, const uint16_t* x, int64_t M, const uin
  * inference the codebook may be quantised uniformly, and it is the 4-bit codebook that speeds the layer
  * up).  q and scale are what cc_quantize_codebook(bits = 4) wrote: ceil(K * g / 2) bytes, element 2k in
  * the low nibble, and one device float.  The weight is the dequantised codebook, value = round-to-nearest-
- * even FP16 of nibble * scale -- exactly the C16_dequantized of cc_quantize_codebook, so the result equals
- * cc_linear_forward on that codebook.  The packed codebook (at most 128 KB: K * g <= 262144) is held in
- * every thread block's shared memory, which turns the gathers from requests to L2 into shared-memory
- * reads.  g even (2..16; other g: CC_ERR_UNSUPPORTED_G); a larger codebook: CC_ERR_SHAPE; q 16-byte
- * aligned; workspace as for cc_linear_forward. */
+ * even FP16 of nibble * scale -- exactly the C16_dequantized of cc_quantize_codebook, so the result is
+ * that of cc_linear_forward on that codebook (bit for bit for 5 <= M <= 64, where both take the same
+ * tensor-core route; otherwise up to the order of the FP32 additions).  The packed codebook (at most
+ * 128 KB: K * g <= 262144) is held in every thread block's shared memory, which turns the gathers from
+ * requests to L2 into shared-memory reads.  For a handful of tokens (M <= 4; M <= 2 when g > 8) a
+ * kernel without the tensor core runs: table look-ups and FP32 multiply-adds, partial sums added in a
+ * fixed order (the same bits on every call).  g even (2..16; other g: CC_ERR_UNSUPPORTED_G); a larger
+ * codebook: CC_ERR_SHAPE; q 16-byte aligned; workspace as for cc_linear_forward.  Calls on one context
+ * must not overlap on the device (they share the workspace and its counters). */
 cc_status cc_linear_forward_q4(cc_ctx* ctx, const uint16_t* x, int64_t M, const uint8_t* q, const float* scale, int K,
                                int g, const uint16_t* idx, int64_t d_out, int64_t d_in, const float* bias, float* y,
                                void* stream);

@@ -57,7 +57,9 @@ struct ProfScope {
 
 // Carving of the workspace for a problem (N, g, K).  All offsets 256-byte aligned.
 struct WsLayout {
-    size_t status;     // 64 x u32: [0] status bits, [2..3] flagged counter (u64)
+    size_t status;     // 64 x u32: [0] status bits, [2..3] flagged counter (u64), [8] last-block counter of the objective
+                       // sum, [32..35] tensor-path parameters, [36] codebook quantiser's maximum, [40..63] arrival
+                       // counters of the few-token layer forward (zero between calls)
     size_t cprep;      // staged codebook for the FFMA E-step
     size_t flagged;    // u32 list of points sent to the exact stage
     size_t partials;   // doubles: per-block objective partial sums

@@ -164,7 +164,7 @@ split_empty_kernel(float* __restrict__ C, int K, int g, const int* __restrict__ 
 
 cudaError_t cc_launch_quantize_codebook(cc_ctx* ctx, const uint16_t* C16, int64_t n, int bits, uint8_t* q, float* scale,
                                         uint16_t* deq, cudaStream_t st) {
-    unsigned* max_bits = reinterpret_cast<unsigned*>(static_cast<char*>(ctx->ws) + 192);   // spare status word
+    unsigned* max_bits = reinterpret_cast<unsigned*>(static_cast<char*>(ctx->ws) + 144);   // word 36 of the status block
     cudaError_t e = cudaMemsetAsync(max_bits, 0, sizeof(unsigned), st);
     if (e != cudaSuccess) return e;
     {

@@ -93,6 +93,7 @@ __device__ __forceinline__ void load_code_row_words(const uint16_t* __restrict__
 // table sits in shared memory, and a 256-entry table turns a byte into its two dequantised FP16 values
 // (value = round-to-nearest-even FP16 of nibble * scale, the nibble a two's-complement number).
 constexpr int LQ_TABLE_MAX = 128 * 1024;   // bytes of packed codebook that fit beside the stages
+constexpr int LQ_BULK_PIECE = 32 * 1024;   // bytes per bulk copy of the table
 constexpr int LQ_NT_MAX = 64;              // tokens per CTA when the table takes most of the shared memory
 
 template <int G>
@@ -122,6 +123,7 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
     uint64_t* full = bars, *empty = bars + LSTAGES, *acc_full = bars + 2 * LSTAGES;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * LSTAGES + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
+    uint64_t* qbar = bars + 16;                                                                  // QUANT only: the table has landed
     uint32_t* lut2 = reinterpret_cast<uint32_t*>(reinterpret_cast<unsigned char*>(bars) + 256);   // QUANT only
     unsigned char* qt = reinterpret_cast<unsigned char*>(lut2 + 256);                            // QUANT only
 
@@ -140,8 +142,24 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(empty + s)));
         }
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(acc_full)));
+        if constexpr (QUANT) asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(qbar)));
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        if constexpr (QUANT) {
+            // the packed codebook comes in as bulk copies (whole 16-byte pieces; the threads fetch the rest below)
+            // while the CTA sets itself up; the producers wait for it before their first look-up
+            const uint32_t bulk = (uint32_t)(K * (G / 2)) & ~15u, bar = smem_u32(qbar);
+            if (bulk) {
+                asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bulk) : "memory");
+                for (uint32_t off = 0; off < bulk; off += LQ_BULK_PIECE) {
+                    const uint32_t n = bulk - off < (uint32_t)LQ_BULK_PIECE ? bulk - off : (uint32_t)LQ_BULK_PIECE;
+                    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                                 ::"r"(smem_u32(qt + off)), "l"(qtab + off), "r"(n), "r"(bar) : "memory");
+                }
+            } else {
+                asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+            }
+        }
     }
     if (warp == 0) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(tmem_slot)),
@@ -158,8 +176,6 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
             lut2[tid] = a | (b << 16);
         }
         const int bytes = K * (G / 2);
-        for (int v = tid; v < bytes / 16; v += LTHREADS)
-            reinterpret_cast<uint4*>(qt)[v] = __ldg(reinterpret_cast<const uint4*>(qtab) + v);
         for (int v = (bytes / 16) * 16 + tid; v < bytes; v += LTHREADS) qt[v] = __ldg(qtab + v);
     }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -176,6 +192,7 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
         const int n_grp = grp_hi - grp_lo + 1;                      // >= 1: o0 < d_out <= out_groups * G
         const bool vec_x = (d_in % 8) == 0;
         bool ok = true;
+        if constexpr (QUANT) ok = mbar_wait(smem_u32(qbar), 0, abort_flag);
         const int st = tid / LSTAGE_THREADS;                        // the stage this thread's group of warps fills
         const int ptid = tid - st * LSTAGE_THREADS;
         for (int c = st; c < n_chunks && ok; c += LSTAGES) {
@@ -360,6 +377,12 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
         }
     }
     if (*abort_flag && lane == 0) atomicOr(status, CC_DEV_TIMEOUT);
+    if constexpr (QUANT) {
+        if (*abort_flag && tid == 0) {   // let the table's copies land before the CTA gives its shared memory back (bounded)
+            const long long t0 = clock64();
+            while (!mbar_try(smem_u32(qbar), 0) && clock64() - t0 < WAIT_LIMIT) {}
+        }
+    }
     asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
     __syncthreads();
     if (warp == 0)
@@ -375,6 +398,212 @@ linear_reduce_kernel(const float* __restrict__ partial, int splits, int64_t n, i
         for (int k = 0; k < splits; ++k) s += partial[(int64_t)k * n + e];
         y[e] = s;
     }
+}
+
+// ---- A handful of tokens (M <= 4; M <= 2 for g > 8) on the 4-bit codebook: no tensor core.  With so few columns the MMA
+// idles and the tensor kernel's time is its producers' instructions; here a thread owns one code group (g
+// out_features), walks down the in_features of its CTA's slice, looks each code up in the packed table in
+// shared memory (one load of g / 2 bytes, then one load per 4-bit level from a 16-entry FP32 table, whose
+// entries lie in 16 different banks: no conflicts whatever the levels) and adds x times the g values
+// to M x g FP32 accumulators.  A product of two FP16 values is exact in FP32, so only the additions round.
+// CTA = 64 code groups x 16 interleaved sub-slices of the in_features; the sixteen partial sums meet in
+// shared memory in a fixed order, and the CTA writes its slab of partial sums (y itself when the layer
+// needs a single slice per block of code groups); the slabs are added in slice order by the CTA that
+// finishes last, or by linear_reduce_kernel: the same bits on every call.
+// blockIdx.x: block of 64 code groups; blockIdx.y: slice of rows_per_split in_features.
+constexpr int LG_THREADS = 1024, LG_GRPS = 64, LG_SUB = 16, LG_ROWS_MAX = 1024, LG_M_MAX = 4;
+constexpr int LG_COUNTER_WORD = 40, LG_COUNTERS = 24;   // words 40..63 of the 64-word status block
+
+template <int G>
+__device__ __forceinline__ void gemv_levels(const unsigned char* row, unsigned (&lv)[G]) {
+    if constexpr (G == 4) {
+        const unsigned w = *reinterpret_cast<const uint16_t*>(row);
+#pragma unroll
+        for (int t = 0; t < 4; ++t) lv[t] = (w >> (4 * t)) & 15u;
+    } else if constexpr (G == 8) {
+        const unsigned w = *reinterpret_cast<const unsigned*>(row);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) lv[t] = (w >> (4 * t)) & 15u;
+    } else if constexpr (G == 16) {
+        const uint2 w = *reinterpret_cast<const uint2*>(row);
+#pragma unroll
+        for (int t = 0; t < 8; ++t) { lv[t] = (w.x >> (4 * t)) & 15u; lv[8 + t] = (w.y >> (4 * t)) & 15u; }
+    } else {
+#pragma unroll
+        for (int b = 0; b < G / 2; ++b) { const unsigned w = row[b]; lv[2 * b] = w & 15u; lv[2 * b + 1] = w >> 4; }
+    }
+}
+
+template <int G, int MT>
+__global__ void __launch_bounds__(LG_THREADS, 1)
+linear_gemv_q4_kernel(const uint16_t* __restrict__ x, int M, const unsigned char* __restrict__ qtab,
+                      const float* __restrict__ qscale, int K, const uint16_t* __restrict__ idx, int d_out, int d_in,
+                      int out_groups, int rows_per_split, float* __restrict__ out, int64_t split_stride,
+                      unsigned* __restrict__ status, unsigned* __restrict__ arrived, const float* __restrict__ bias,
+                      float* __restrict__ y, int direct) {
+    extern __shared__ __align__(16) unsigned char gv_smem[];
+    uint64_t* qbar = reinterpret_cast<uint64_t*>(gv_smem);                       // the table has landed
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(gv_smem + 8);
+    float* lut16 = reinterpret_cast<float*>(gv_smem + 64);                       // level -> value
+    float* xs = reinterpret_cast<float*>(gv_smem + 128);                         // [row][MT]
+    unsigned char* qt = gv_smem + 128 + ((size_t)rows_per_split * MT * 4 + 15) / 16 * 16;   // packed table, later the exchange area
+    const int tid = threadIdx.x, gl = tid % LG_GRPS, sub = tid / LG_GRPS;
+    const int i0 = blockIdx.y * rows_per_split;
+    int rows = d_in - i0;
+    rows = rows < rows_per_split ? rows : rows_per_split;
+    const int bytes = K * (G / 2);
+    if (tid == 0) {
+        asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(qbar)));
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        const uint32_t bulk = (uint32_t)bytes & ~15u, bar = smem_u32(qbar);
+        if (bulk) {
+            asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bulk) : "memory");
+            for (uint32_t off = 0; off < bulk; off += LQ_BULK_PIECE) {
+                const uint32_t n = bulk - off < (uint32_t)LQ_BULK_PIECE ? bulk - off : (uint32_t)LQ_BULK_PIECE;
+                asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                             ::"r"(smem_u32(qt + off)), "l"(qtab + off), "r"(n), "r"(bar) : "memory");
+            }
+        } else {
+            asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+        }
+    }
+    for (int v = (bytes / 16) * 16 + tid; v < bytes; v += LG_THREADS) qt[v] = __ldg(qtab + v);
+    if (tid < 16) {
+        const int level = (tid ^ 8) - 8;                                         // sign-extended
+        lut16[tid] = __half2float(__float2half_rn(__fmul_rn((float)level, __ldg(qscale))));   // the quantiser's own value
+    }
+    for (int e = tid; e < rows * MT; e += LG_THREADS) {
+        const int r = e / MT, m = e - r * MT;
+        xs[e] = (m < M) ? __half2float(__ushort_as_half(__ldg(x + (int64_t)m * d_in + i0 + r))) : 0.f;
+    }
+    __syncthreads();
+    bool ok = true, waited = false;                        // the first codes are requested before the wait for the table
+
+    const int grp = blockIdx.x * LG_GRPS + gl;
+    const bool live = grp < out_groups;
+    float acc[MT][G];
+#pragma unroll
+    for (int m = 0; m < MT; ++m)
+#pragma unroll
+        for (int t = 0; t < G; ++t) acc[m][t] = 0.f;
+    const unsigned kmax = (unsigned)K - 1u;
+    if (live) {
+        const uint16_t* col = idx + (int64_t)i0 * out_groups + grp;
+        constexpr int RB = 4;                                                    // rows whose codes are requested together
+        for (int r0 = sub; r0 < rows; r0 += RB * LG_SUB) {
+            unsigned code[RB];
+#pragma unroll
+            for (int u = 0; u < RB; ++u) {
+                const int r = r0 + u * LG_SUB;
+                code[u] = (r < rows) ? (unsigned)__ldg(col + (int64_t)r * out_groups) : 0u;
+            }
+            if (!waited) {
+                ok = mbar_wait(smem_u32(qbar), 0, abort_flag);
+                waited = true;
+                if (!ok) break;
+            }
+#pragma unroll
+            for (int u = 0; u < RB; ++u) {
+                const int r = r0 + u * LG_SUB;
+                if (r >= rows) break;
+                unsigned lv[G];
+                gemv_levels<G>(qt + (size_t)min(code[u], kmax) * (G / 2), lv);   // a code beyond the codebook must not leave it
+                float xv[MT];
+#pragma unroll
+                for (int m = 0; m < MT; ++m) xv[m] = xs[r * MT + m];
+#pragma unroll
+                for (int t = 0; t < G; ++t) {
+                    const float c = lut16[lv[t]];
+#pragma unroll
+                    for (int m = 0; m < MT; ++m) acc[m][t] = fmaf(xv[m], c, acc[m][t]);
+                }
+            }
+        }
+    }
+    if (!waited) ok = mbar_wait(smem_u32(qbar), 0, abort_flag);   // nobody writes over the table's place before it has landed
+    // ---- the sub-slices meet, one token at a time (the exchange area takes the table's place)
+    __syncthreads();
+    float* red = reinterpret_cast<float*>(qt);                                   // [LG_SUB - 1][G][LG_GRPS]
+    float* dst = out + (int64_t)blockIdx.y * split_stride;
+#pragma unroll
+    for (int m = 0; m < MT; ++m) {
+        if (sub > 0) {
+#pragma unroll
+            for (int t = 0; t < G; ++t) red[((sub - 1) * G + t) * LG_GRPS + gl] = acc[m][t];
+        }
+        __syncthreads();
+        if (sub == 0 && m < M && grp < out_groups && !*abort_flag) {
+#pragma unroll
+            for (int t = 0; t < G; ++t) {
+                float s = acc[m][t];
+#pragma unroll
+                for (int q = 0; q < LG_SUB - 1; ++q) s += red[(q * G + t) * LG_GRPS + gl];
+                const int o = grp * G + t;
+                if (o < d_out) dst[(int64_t)m * d_out + o] = (direct && bias) ? s + __ldg(bias + o) : s;
+            }
+        }
+        __syncthreads();
+    }
+    if (*abort_flag && tid == 0) {
+        atomicOr(status, CC_DEV_TIMEOUT);
+        const long long t0 = clock64();                                          // let the table's copies land (bounded)
+        while (!mbar_try(smem_u32(qbar), 0) && clock64() - t0 < WAIT_LIMIT) {}
+    }
+    // ---- the CTA that finishes last among the slices of this block of code groups adds the slabs, in slice
+    // order (the same bits whichever CTA that is), and the bias; it leaves the counter at zero for the next call.
+    // Every CTA counts itself, also one that gave up, so that the counter always returns to zero.
+    if (arrived) {
+        __shared__ int last;
+        __threadfence();                                                         // this thread's slab stores before the count
+        __syncthreads();
+        if (tid == 0) last = atomicAdd(arrived + blockIdx.x, 1u) == gridDim.y - 1;
+        __syncthreads();
+        if (last) {
+            __threadfence();
+            const int o_lo = blockIdx.x * LG_GRPS * G;
+            int width = d_out - o_lo;
+            width = width < LG_GRPS * G ? width : LG_GRPS * G;
+            for (int e = tid; e < M * width; e += LG_THREADS) {
+                const int m = e / width, o = o_lo + (e - m * width);
+                const float* src = out + (int64_t)m * d_out + o;
+                float sum = bias ? __ldg(bias + o) : 0.f;
+                unsigned k = 0;
+                for (; k + 8 <= gridDim.y; k += 8) {                             // eight loads in flight, added in slice order
+                    float v[8];
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) v[u] = __ldcg(src + (int64_t)(k + u) * split_stride);
+#pragma unroll
+                    for (int u = 0; u < 8; ++u) sum += v[u];
+                }
+                for (; k < gridDim.y; ++k) sum += __ldcg(src + (int64_t)k * split_stride);
+                y[(int64_t)m * d_out + o] = sum;
+            }
+            if (tid == 0) arrived[blockIdx.x] = 0u;
+        }
+    }
+}
+
+struct GemvPlan { int o_blocks, splits, rows_per_split; };
+
+GemvPlan gemv_plan(int64_t d_in, int out_groups, int sm_count) {
+    GemvPlan p;
+    p.o_blocks = (out_groups + LG_GRPS - 1) / LG_GRPS;
+    int splits = sm_count / p.o_blocks;                                          // one CTA per SM where the shape allows
+    if (splits < 1) splits = 1;
+    if ((int64_t)splits * 16 > d_in) splits = (int)((d_in + 15) / 16);           // at least 16 in_features per CTA
+    int64_t rows = (d_in + splits - 1) / splits;
+    if (rows > LG_ROWS_MAX) rows = LG_ROWS_MAX;
+    p.rows_per_split = (int)rows;
+    p.splits = (int)((d_in + rows - 1) / rows);
+    return p;
+}
+
+size_t gemv_smem(int g, int K, int rows, int mt) {
+    size_t tail = (size_t)K * (g / 2);
+    const size_t red = (size_t)(LG_SUB - 1) * g * LG_GRPS * 4;
+    if (tail < red) tail = red;
+    return 128 + ((size_t)rows * mt * 4 + 15) / 16 * 16 + (tail + 15) / 16 * 16;
 }
 
 struct LinearPlan { int NT, tmem_cols, o_tiles, tok_blocks, splits, chunks_per_split; size_t smem; };
@@ -405,8 +634,15 @@ size_t cc_linear_scratch_bytes(int64_t M, int64_t d_out, int64_t d_in, int sm_co
     // enough for either form of the codebook: the quantised one takes narrower token blocks and may split more
     const LinearPlan p = linear_plan(M, d_out, d_in, sm_count);
     const LinearPlan q = linear_plan(M, d_out, d_in, sm_count, LQ_NT_MAX, 16);
-    const int splits = p.splits > q.splits ? p.splits : q.splits;
-    return 256 + (splits > 1 ? (size_t)splits * (size_t)M * (size_t)d_out * 4 : 0);
+    int splits = p.splits > q.splits ? p.splits : q.splits;
+    if (splits < 2) splits = 0;    // a single CTA per tile writes y itself
+    if (M <= LG_M_MAX) {
+        // the few-token kernel of the quantised codebook always goes through its slabs; the most slices come
+        // with the fewest blocks of code groups, i.e. at g = 16
+        const GemvPlan v = gemv_plan(d_in, (int)((d_out + 15) / 16), sm_count);
+        if (v.splits > splits) splits = v.splits;
+    }
+    return 256 + (size_t)splits * (size_t)M * (size_t)d_out * 4;
 }
 
 int cc_linear_q_table_max(void) { return LQ_TABLE_MAX; }
@@ -448,6 +684,49 @@ cudaError_t launch_linear(cc_ctx* ctx, const LinearPlan& p, const uint16_t* x, i
 
 }  // namespace
 
+namespace {
+
+template <int G, int MT>
+cudaError_t launch_gemv(cc_ctx* ctx, const GemvPlan& p, const uint16_t* x, int M, const unsigned char* qtab,
+                        const float* qscale, int K, const uint16_t* idx, int d_out, int d_in, int out_groups, float* out,
+                        int64_t split_stride, unsigned* status, unsigned* arrived, const float* bias, float* y,
+                        cudaStream_t st) {
+    static bool attr_dev[64] = {};
+    bool& have = attr_dev[ctx->device & 63];
+    if (!have) {
+        const cudaError_t e = cudaFuncSetAttribute(linear_gemv_q4_kernel<G, MT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                   (int)gemv_smem(G, LQ_TABLE_MAX / (G / 2), LG_ROWS_MAX, MT));
+        if (e != cudaSuccess) return e;
+        have = true;
+    }
+    const dim3 grid(p.o_blocks, p.splits);
+    linear_gemv_q4_kernel<G, MT><<<grid, LG_THREADS, gemv_smem(G, K, p.rows_per_split, MT), st>>>(
+        x, M, qtab, qscale, K, idx, d_out, d_in, out_groups, p.rows_per_split, out, split_stride, status, arrived, bias, y, p.splits == 1);
+    return cudaGetLastError();
+}
+
+// Tokens padded to 1, 2 or 4 (from 8 on the tensor kernel is as fast); M x g accumulators must fit the
+// registers of 1024 threads per SM.
+constexpr int gemv_tokens(int g) { return g <= 8 ? 4 : 2; }
+
+template <int G>
+cudaError_t launch_gemv_m(cc_ctx* ctx, const GemvPlan& p, const uint16_t* x, int M, const unsigned char* qtab,
+                          const float* qscale, int K, const uint16_t* idx, int d_out, int d_in, int out_groups, float* out,
+                          int64_t split_stride, unsigned* status, unsigned* arrived, const float* bias, float* y,
+                          cudaStream_t st) {
+    if (M == 1) return launch_gemv<G, 1>(ctx, p, x, M, qtab, qscale, K, idx, d_out, d_in, out_groups, out, split_stride, status, arrived, bias, y, st);
+    if (M == 2) return launch_gemv<G, 2>(ctx, p, x, M, qtab, qscale, K, idx, d_out, d_in, out_groups, out, split_stride, status, arrived, bias, y, st);
+    if constexpr (gemv_tokens(G) >= 4) {
+        if (M <= 4) return launch_gemv<G, 4>(ctx, p, x, M, qtab, qscale, K, idx, d_out, d_in, out_groups, out, split_stride, status, arrived, bias, y, st);
+    }
+    if constexpr (gemv_tokens(G) >= 8) {
+        if (M <= 8) return launch_gemv<G, 8>(ctx, p, x, M, qtab, qscale, K, idx, d_out, d_in, out_groups, out, split_stride, status, arrived, bias, y, st);
+    }
+    return cudaErrorInvalidValue;
+}
+
+}  // namespace
+
 // qtab == nullptr: FP16 codebook C16; otherwise the packed 4-bit codebook with its scale (even g only).
 cudaError_t cc_launch_linear_forward(cc_ctx* ctx, const uint16_t* x, int64_t M, const uint16_t* C16,
                                      const unsigned char* qtab, const float* qscale, int K, int g, const uint16_t* idx,
@@ -460,6 +739,33 @@ cudaError_t cc_launch_linear_forward(cc_ctx* ctx, const uint16_t* x, int64_t M, 
     const int out_groups = (int)((d_out + g - 1) / g);
     const int64_t n = M * d_out;
     cudaError_t e = cudaSuccess;
+    if (qtab && M <= gemv_tokens(g)) {
+        // a handful of tokens: the shared-memory look-up kernel, then the same reduction (it also adds the bias)
+        const GemvPlan v = gemv_plan(d_in, out_groups, ctx->sm_count);
+        unsigned* arrived = nullptr;
+        {
+            ProfScope ps(ctx, CC_K_LINEAR, st);
+            // counters of the finished slices: words of the status block that nothing else uses (zero since
+            // cc_set_workspace, put back to zero by the kernel); with more blocks than counters the reduction
+            // is a kernel of its own
+            arrived = (v.splits > 1 && v.o_blocks <= LG_COUNTERS) ? status + LG_COUNTER_WORD : nullptr;
+            float* slabs = v.splits == 1 ? y : partial;          // a single slice writes y (and the bias) itself
+#define CALL(G) e = launch_gemv_m<G>(ctx, v, x, (int)M, qtab, qscale, K, idx, (int)d_out, (int)d_in, out_groups, slabs, n, status, arrived, bias, y, st)
+            switch (g) {
+                case 2: CALL(2); break;   case 4: CALL(4); break;   case 6: CALL(6); break;   case 8: CALL(8); break;
+                case 10: CALL(10); break; case 12: CALL(12); break; case 14: CALL(14); break; case 16: CALL(16); break;
+                default: return cudaErrorInvalidValue;
+            }
+#undef CALL
+        }
+        if (e != cudaSuccess || arrived || v.splits == 1) return e;
+        ProfScope ps(ctx, CC_K_LINEAR_REDUCE, st);
+        int64_t blocks = (n + 255) / 256;
+        const int64_t cap = (int64_t)ctx->sm_count * 8;
+        if (blocks > cap) blocks = cap;
+        linear_reduce_kernel<<<(unsigned)blocks, 256, 0, st>>>(partial, v.splits, n, (int)d_out, bias, y);
+        return cudaGetLastError();
+    }
     {
         ProfScope ps(ctx, CC_K_LINEAR, st);
         float* out = p.splits > 1 ? partial : y;

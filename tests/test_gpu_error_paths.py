@@ -52,7 +52,9 @@ class Args:
         self.nres = torch.full((1,), -3, dtype=torch.int64, device="cuda")
         self.scores = torch.full((8, 256), -4.0, dtype=torch.float32, device="cuda")
         self.scan = torch.zeros((N, 2), dtype=torch.float32, device="cuda")
-        self.xin = torch.full((8, D_IN), 0.5, dtype=torch.float16, device="cuda")
+        self.xinbuf = torch.full((8 * D_IN + 8,), 0.5, dtype=torch.float16, device="cuda")
+        self.xin = self.xinbuf[:8 * D_IN].view(8, D_IN)
+        self.xin_odd = self.xinbuf[1:8 * D_IN + 1].view(8, D_IN)
         self.ybuf = torch.full((8 * D_OUT + 8,), -6.0, dtype=torch.float32, device="cuda")
         self.y = self.ybuf[:8 * D_OUT].view(8, D_OUT)
         self.y_odd = self.ybuf[1:8 * D_OUT + 1].view(8, D_OUT)
@@ -107,6 +109,9 @@ def _calls(a, o):
                                           v("d_in", D_IN), v("layout", 0), v("W", a.W)),
         "cc_linear_forward": lambda: cc.cc_linear_forward(ctx, v("x", a.xin), v("M", 8), v("C16", a.C16), v("K", K), v("g", G),
                                                           v("idx", a.idx), v("d_out", D_OUT), v("d_in", D_IN), None, v("y", a.y)),
+        "cc_linear_forward_q4": lambda: cc.cc_linear_forward_q4(ctx, v("x", a.xin), v("M", 8), v("q", a.q8), v("scale", a.scale),
+                                                                v("K", K), v("g", G), v("idx", a.idx), v("d_out", D_OUT),
+                                                                v("d_in", D_IN), None, v("y", a.y)),
         "cc_quantize_codebook": lambda: cc.cc_quantize_codebook(ctx, v("C16", a.C16), v("K", K), v("g", G), v("bits", 8),
                                                                 v("q", a.q8), v("scale", a.scale), a.c16out),
         "cc_fit_sampled": lambda: cc.cc_fit_sampled(ctx, v("X", a.X), v("N", N), v("g", G), v("K", K), v("iters", 1),
@@ -172,6 +177,14 @@ CASES += [
     ("cc_linear_forward", {"idx": None}, NULL), ("cc_linear_forward", {"y": None}, NULL), ("cc_linear_forward", {"M": 0}, SHAPE),
     ("cc_linear_forward", {"d_in": 0}, SHAPE), ("cc_linear_forward", {"M": 1 << 30}, SHAPE),
     ("cc_linear_forward", {"C16": "C16_odd"}, ALIGN), ("cc_linear_forward", {"y": "y_odd"}, ALIGN),
+    ("cc_linear_forward", {"x": "xin_odd"}, ALIGN),
+    ("cc_linear_forward_q4", {"g": 0}, BAD_G), ("cc_linear_forward_q4", {"g": 18}, BAD_G), ("cc_linear_forward_q4", {"g": 3}, BAD_G),
+    ("cc_linear_forward_q4", {"K": 0}, BAD_K), ("cc_linear_forward_q4", {"K": 65537}, BAD_K),
+    ("cc_linear_forward_q4", {"x": None}, NULL), ("cc_linear_forward_q4", {"q": None}, NULL),
+    ("cc_linear_forward_q4", {"scale": None}, NULL), ("cc_linear_forward_q4", {"idx": None}, NULL),
+    ("cc_linear_forward_q4", {"y": None}, NULL), ("cc_linear_forward_q4", {"M": 0}, SHAPE),
+    ("cc_linear_forward_q4", {"d_out": 0}, SHAPE), ("cc_linear_forward_q4", {"y": "y_odd"}, ALIGN),
+    ("cc_linear_forward_q4", {"x": "xin_odd"}, ALIGN),
     ("cc_quantize_codebook", {"g": 0}, BAD_G), ("cc_quantize_codebook", {"K": 65537}, BAD_K),
     ("cc_quantize_codebook", {"bits": 2}, SHAPE), ("cc_quantize_codebook", {"bits": 16}, SHAPE),
     ("cc_quantize_codebook", {"C16": None}, NULL), ("cc_quantize_codebook", {"q": None}, NULL),

@@ -133,10 +133,34 @@ def test_linear_forward_q4_matches_oracle(M, d_out, d_in, g, K):
     want = oracle.linear_forward(x, deq_or, idx.astype(np.int32), d_out, d_in, bias)      # the layer on the dequantised codebook
     _check(y, want)
     y_fp16 = _gpu_forward(x, deq_or, idx, d_out, d_in, bias)                             # the FP16 kernel on the same codebook
-    if M <= 64:            # same token blocks and splits: the same sums in the same order
+    few = 4 if g <= 8 else 2        # up to here the look-up kernel without the tensor core runs
+    if few < M <= 64:      # same token blocks and splits: the same sums in the same order
         assert np.array_equal(y.view(np.uint32), y_fp16.view(np.uint32))
     else:
         _check(y_fp16, want)
+
+
+@pytest.mark.parametrize("M,d_out,d_in,g,K", [
+    (1, 4096, 4096, 4, 65536),      # one token through the paper's largest codebook at g = 4: 37 slices of 111 in_features
+    (4, 4096, 4096, 4, 65536), (3, 1000, 520, 4, 700), (4, 130, 67, 4, 50), (2, 260, 1031, 4, 65535), (2, 28672, 256, 4, 4096),
+    (1, 64, 24, 2, 5), (4, 75, 40, 2, 33), (4, 250, 300, 6, 90), (3, 4096, 2048, 8, 32768), (4, 200, 72, 8, 2900),
+    (2, 144, 328, 10, 77), (1, 260, 64, 12, 300), (2, 300, 96, 14, 19), (2, 2048, 1024, 16, 16384), (1, 8200, 40, 16, 1400),
+    (2, 128, 5000, 4, 256),         # one block of code groups, in_features cut into more slices than 16 each would give
+    (1, 40, 9, 4, 3),               # fewer than 16 in_features
+])
+def test_linear_forward_q4_few_tokens_matches_oracle(M, d_out, d_in, g, K):
+    """The kernel that serves a handful of tokens (no tensor core: table look-ups and FP32 FMAs) against the oracle's
+    layer on the oracle's dequantised codebook; the same bits on every call; with and without bias."""
+    x, C16, idx, bias = _case(M, d_out, d_in, g, K, 7 * M + d_in + g)
+    _, _, deq_or = oracle.quantize_codebook(C16, 4)
+    want = oracle.linear_forward(x, deq_or, idx.astype(np.int32), d_out, d_in, bias)
+    y, _ = _gpu_forward_q4(x, C16, idx, d_out, d_in, bias)
+    worst = _check(y, want)
+    y2, _ = _gpu_forward_q4(x, C16, idx, d_out, d_in, bias)
+    assert np.array_equal(y.view(np.uint32), y2.view(np.uint32))
+    y0, _ = _gpu_forward_q4(x, C16, idx, d_out, d_in, None)
+    _check(y0, want - bias.astype(np.float64))
+    print("M=%d %dx%d g=%d K=%d: worst error %.3f of the bound" % (M, d_out, d_in, g, K, worst))
 
 
 def test_linear_forward_q4_rejects_what_it_cannot_hold():

@@ -35,7 +35,23 @@ constexpr int LPROD = 512;              // producer threads (16 warps); warps 0.
 constexpr int LSTAGE_THREADS = LPROD / LSTAGES;   // producer threads that fill one stage (four warps)
 constexpr int LTHREADS = LPROD + 32;    // + the MMA warp
 constexpr int LNT_MAX = 256;            // tokens per CTA = MMA N
-constexpr int A_STAGE = LM * LKB * 2;   // bytes
+// Operand tiles in shared memory: the K-major no-swizzle layout of 8 x 16-byte core matrices, with the two
+// strides of the descriptor chosen against bank conflicts of the producers' 16-byte stores.  Neighbouring
+// lanes of an A-tile store hold neighbouring code groups, i.e. rows g apart in one column of core matrices:
+// 144 instead of 128 bytes between 8-row groups puts row r at 16-byte slot 9 (r / 8) + r % 8, and the eight
+// lanes of a store phase then fall into eight different slots mod 8 for g = 2, 4, 8 (two by two for g = 16;
+// at 128 bytes they all shared one or two).  Neighbouring lanes of a B-tile store hold neighbouring
+// 8-column pieces of one token's row: 16 bytes more between the columns of core matrices does the same.
+// Measured (4096 x 4096, g 4, K 65536): the B stride alone 0.772 -> 0.585 ms at 4096 tokens, 64 -> 50 us at
+// 256; the A stride on top 35.7 -> 33.6 us at 64 tokens (87 -> 64 us at g = 8 on 8192 x 8192, 16 tokens) but
+// 0.585 -> 0.807 ms at 4096 tokens, where the MMA's own reads of the wider-spaced A tile come to matter:
+// the A tile is widened for token blocks of at most 64 only, and never beside the 4-bit table (no room).
+__host__ __device__ constexpr int a_sbo(bool pad) { return pad ? 144 : 128; }
+__host__ __device__ constexpr int a_lbo(bool pad) { return (LM / 8) * a_sbo(pad); }
+__host__ __device__ constexpr int a_stage(bool pad) { return (LKB / 8) * a_lbo(pad); }   // bytes
+__host__ __device__ constexpr int b_lbo(int nt) { return nt * 16 + 16; }
+__host__ __device__ constexpr int b_stage_bytes(int nt) { return (LKB / 8) * b_lbo(nt); }
+__device__ __forceinline__ int tile_off(int r, int kc, int lbo, int sbo) { return kc * lbo + (r >> 3) * sbo + (r & 7) * 16; }
 
 // Row of G halves of the codebook as raw bit patterns.
 template <int G>
@@ -113,10 +129,11 @@ __global__ void __launch_bounds__(LTHREADS, 1)
 linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __restrict__ C16,
                       const unsigned char* __restrict__ qtab, const float* __restrict__ qscale, int K,
                       const uint16_t* __restrict__ idx, int d_out, int d_in, int out_groups, int NT,
-                      int tmem_cols, int chunks_per_split, float* __restrict__ out, int64_t split_stride,
+                      int a_pad, int tmem_cols, int chunks_per_split, float* __restrict__ out, int64_t split_stride,
                       const float* __restrict__ bias, unsigned* __restrict__ status) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
-    const int b_stage = NT * LKB * 2;
+    const int A_STAGE = a_stage(a_pad), A_LBO = a_lbo(a_pad), A_SBO = a_sbo(a_pad);
+    const int b_stage = b_stage_bytes(NT), B_LBO = b_lbo(NT);
     unsigned char* sA = smem_raw;                                   // LSTAGES tiles of 128 x 64
     unsigned char* sB = sA + LSTAGES * A_STAGE;                     // LSTAGES tiles of NT x 64
     uint64_t* bars = reinterpret_cast<uint64_t*>(sB + LSTAGES * b_stage);
@@ -249,7 +266,7 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
                             w.y = __byte_perm(v[q][2][t / 2], v[q][3][t / 2], sel);
                             w.z = __byte_perm(v[q][4][t / 2], v[q][5][t / 2], sel);
                             w.w = __byte_perm(v[q][6][t / 2], v[q][7][t / 2], sel);
-                            *reinterpret_cast<uint4*>(tA + canon_bytes(r, ibs[q] * 8, LM)) = w;
+                            *reinterpret_cast<uint4*>(tA + tile_off(r, ibs[q], A_LBO, A_SBO)) = w;
                         }
                     }
                 } else {
@@ -279,7 +296,7 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
                         w.y = (unsigned)v[2][t] | ((unsigned)v[3][t] << 16);
                         w.z = (unsigned)v[4][t] | ((unsigned)v[5][t] << 16);
                         w.w = (unsigned)v[6][t] | ((unsigned)v[7][t] << 16);
-                        *reinterpret_cast<uint4*>(tA + canon_bytes(r, ib * 8, LM)) = w;
+                        *reinterpret_cast<uint4*>(tA + tile_off(r, ib, A_LBO, A_SBO)) = w;
                     }
                 }
             }
@@ -313,7 +330,7 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
                     const int item = item0 + u4 * LSTAGE_THREADS;
                     if (item < n_b) {
                         const int kc = item % (LKB / 8), r = item / (LKB / 8);
-                        *reinterpret_cast<uint4*>(tB + canon_bytes(r, kc * 8, NT)) = w[u4];
+                        *reinterpret_cast<uint4*>(tB + tile_off(r, kc, B_LBO, 128)) = w[u4];
                     }
                 }
             }
@@ -346,8 +363,8 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
         if (lane == 0) {
             // kind::f16: D = F32 (bits 4-5 = 1), A = B = F16 (0), both K-major, N >> 3 at bit 17, M >> 4 at bit 24
             const uint32_t idesc = (1u << 4) | ((uint32_t)(NT >> 3) << 17) | ((uint32_t)(LM >> 4) << 24);
-            const uint64_t descA0 = make_desc(smem_u32(sA), LM * 16, 128);
-            const uint64_t descB0 = make_desc(smem_u32(sB), NT * 16, 128);
+            const uint64_t descA0 = make_desc(smem_u32(sA), A_LBO, A_SBO);
+            const uint64_t descB0 = make_desc(smem_u32(sB), B_LBO, 128);
             bool ok = true;
             for (int c = 0; c < n_chunks && ok; ++c) {
                 const int st = c % LSTAGES;
@@ -358,8 +375,8 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
                 const uint64_t descB = descB0 + (uint64_t)((st * b_stage) >> 4);
 #pragma unroll
                 for (int s = 0; s < LKB / 16; ++s) {
-                    const uint64_t da = descA + (uint64_t)((s * 2 * (LM * 16)) >> 4);
-                    const uint64_t db = descB + (uint64_t)((s * 2 * (NT * 16)) >> 4);
+                    const uint64_t da = descA + (uint64_t)((s * 2 * A_LBO) >> 4);
+                    const uint64_t db = descB + (uint64_t)((s * 2 * B_LBO) >> 4);
                     const uint32_t acc = (c > 0 || s > 0) ? 1u : 0u;
                     asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
                                  "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
@@ -606,7 +623,7 @@ size_t gemv_smem(int g, int K, int rows, int mt) {
     return 128 + ((size_t)rows * mt * 4 + 15) / 16 * 16 + (tail + 15) / 16 * 16;
 }
 
-struct LinearPlan { int NT, tmem_cols, o_tiles, tok_blocks, splits, chunks_per_split; size_t smem; };
+struct LinearPlan { int NT, a_pad, tmem_cols, o_tiles, tok_blocks, splits, chunks_per_split; size_t smem; };
 
 // nt_max: tokens per CTA (256, or 64 with a quantised codebook in shared memory); table_bytes: that codebook.
 LinearPlan linear_plan(int64_t M, int64_t d_out, int64_t d_in, int sm_count, int nt_max = LNT_MAX, size_t table_bytes = 0) {
@@ -623,7 +640,8 @@ LinearPlan linear_plan(int64_t M, int64_t d_out, int64_t d_in, int sm_count, int
     if (splits < 1) splits = 1;
     p.chunks_per_split = (chunks + splits - 1) / splits;
     p.splits = (chunks + p.chunks_per_split - 1) / p.chunks_per_split;
-    p.smem = (size_t)LSTAGES * (A_STAGE + (size_t)p.NT * LKB * 2) + 256;
+    p.a_pad = (table_bytes == 0 && p.NT <= 64) ? 1 : 0;
+    p.smem = (size_t)LSTAGES * (a_stage(p.a_pad) + (size_t)b_stage_bytes(p.NT)) + 256;
     if (table_bytes) p.smem += 1024 + (table_bytes + 15) / 16 * 16;
     return p;
 }
@@ -668,8 +686,8 @@ cudaError_t launch_linear(cc_ctx* ctx, const LinearPlan& p, const uint16_t* x, i
     static bool attr_dev[64] = {};
     bool& have = attr_dev[ctx->device & 63];
     if (!have) {
-        const int max_smem = QUANT ? (int)(LSTAGES * (A_STAGE + LQ_NT_MAX * LKB * 2) + 256 + 1024 + LQ_TABLE_MAX)
-                                   : (int)(LSTAGES * (A_STAGE + LNT_MAX * LKB * 2) + 256);
+        const int max_smem = QUANT ? (int)(LSTAGES * (a_stage(false) + b_stage_bytes(LQ_NT_MAX)) + 256 + 1024 + LQ_TABLE_MAX)
+                                   : (int)(LSTAGES * (a_stage(true) + b_stage_bytes(LNT_MAX)) + 256);
         const cudaError_t e = cudaFuncSetAttribute(linear_forward_kernel<G, QUANT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                    max_smem);
         if (e != cudaSuccess) return e;
@@ -677,7 +695,7 @@ cudaError_t launch_linear(cc_ctx* ctx, const LinearPlan& p, const uint16_t* x, i
     }
     const dim3 grid(p.o_tiles, p.tok_blocks, p.splits);
     linear_forward_kernel<G, QUANT><<<grid, LTHREADS, p.smem, st>>>(x, M, C16, qtab, qscale, K, idx, d_out, d_in, out_groups,
-                                                                    p.NT, p.tmem_cols, p.chunks_per_split, out, split_stride,
+                                                                    p.NT, p.a_pad, p.tmem_cols, p.chunks_per_split, out, split_stride,
                                                                     bias, status);
     return cudaGetLastError();
 }

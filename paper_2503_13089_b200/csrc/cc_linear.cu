@@ -30,9 +30,8 @@ namespace {
 
 constexpr int LM = 128;                 // out_features per CTA = MMA M = TMEM lanes
 constexpr int LKB = 64;                 // in_features per pipeline stage
-constexpr int LSTAGES = 4;
+constexpr int LSTAGES = 4;              // at most; two where the 4-bit table leaves room for no more wide tiles
 constexpr int LPROD = 512;              // producer threads (16 warps); warps 0..3 also run the epilogue
-constexpr int LSTAGE_THREADS = LPROD / LSTAGES;   // producer threads that fill one stage (four warps)
 constexpr int LTHREADS = LPROD + 32;    // + the MMA warp
 constexpr int LNT_MAX = 256;            // tokens per CTA = MMA N
 // Operand tiles in shared memory: the K-major no-swizzle layout of 8 x 16-byte core matrices, with the two
@@ -110,6 +109,7 @@ __device__ __forceinline__ void load_code_row_words(const uint16_t* __restrict__
 // (value = round-to-nearest-even FP16 of nibble * scale, the nibble a two's-complement number).
 constexpr int LQ_TABLE_MAX = 128 * 1024;   // bytes of packed codebook that fit beside the stages
 constexpr int LQ_BULK_PIECE = 32 * 1024;   // bytes per bulk copy of the table
+constexpr int LQ_WIDE_FROM = 256;
 constexpr int LQ_NT_MAX = 64;              // tokens per CTA when the table takes most of the shared memory
 
 template <int G>
@@ -129,14 +129,15 @@ __global__ void __launch_bounds__(LTHREADS, 1)
 linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __restrict__ C16,
                       const unsigned char* __restrict__ qtab, const float* __restrict__ qscale, int K,
                       const uint16_t* __restrict__ idx, int d_out, int d_in, int out_groups, int NT,
-                      int a_pad, int tmem_cols, int chunks_per_split, float* __restrict__ out, int64_t split_stride,
+                      int a_pad, int n_stages, int tmem_cols, int chunks_per_split, float* __restrict__ out, int64_t split_stride,
                       const float* __restrict__ bias, unsigned* __restrict__ status) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     const int A_STAGE = a_stage(a_pad), A_LBO = a_lbo(a_pad), A_SBO = a_sbo(a_pad);
     const int b_stage = b_stage_bytes(NT), B_LBO = b_lbo(NT);
-    unsigned char* sA = smem_raw;                                   // LSTAGES tiles of 128 x 64
-    unsigned char* sB = sA + LSTAGES * A_STAGE;                     // LSTAGES tiles of NT x 64
-    uint64_t* bars = reinterpret_cast<uint64_t*>(sB + LSTAGES * b_stage);
+    unsigned char* sA = smem_raw;                                   // n_stages (2 or 4) tiles of 128 x 64
+    unsigned char* sB = sA + n_stages * A_STAGE;                    // n_stages tiles of NT x 64
+    uint64_t* bars = reinterpret_cast<uint64_t*>(sB + n_stages * b_stage);
+    const int stage_threads = LPROD / n_stages;                     // producer threads that fill one stage
     uint64_t* full = bars, *empty = bars + LSTAGES, *acc_full = bars + 2 * LSTAGES;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * LSTAGES + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -154,8 +155,8 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
     if (n_chunks < 0) n_chunks = 0;
 
     if (tid == 0) {
-        for (int s = 0; s < LSTAGES; ++s) {
-            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(full + s)), "r"(LSTAGE_THREADS));
+        for (int s = 0; s < n_stages; ++s) {
+            asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(full + s)), "r"(stage_threads));
             asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(empty + s)));
         }
         asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(smem_u32(acc_full)));
@@ -210,10 +211,10 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
         const bool vec_x = (d_in % 8) == 0;
         bool ok = true;
         if constexpr (QUANT) ok = mbar_wait(smem_u32(qbar), 0, abort_flag);
-        const int st = tid / LSTAGE_THREADS;                        // the stage this thread's group of warps fills
-        const int ptid = tid - st * LSTAGE_THREADS;
-        for (int c = st; c < n_chunks && ok; c += LSTAGES) {
-            ok = mbar_wait(smem_u32(empty + st), ((c / LSTAGES) & 1) ^ 1, abort_flag);
+        const int st = tid / stage_threads;                         // the stage this thread's group of warps fills
+        const int ptid = tid - st * stage_threads;
+        for (int c = st; c < n_chunks && ok; c += n_stages) {
+            ok = mbar_wait(smem_u32(empty + st), ((c / n_stages) & 1) ^ 1, abort_flag);
             if (!ok) break;
             unsigned char* tA = sA + st * A_STAGE;
             unsigned char* tB = sB + st * b_stage;
@@ -222,7 +223,7 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
             // IPT items per thread and pass: all their codes are requested first, then all their rows, so that a
             // pass costs two trips to L2 whatever IPT is (the rows of IPT items must fit the registers)
             constexpr int IPT = (G % 2 == 0 && G <= 8) ? 2 : 1;
-            for (int item0 = ptid; item0 < (LKB / 8) * n_grp; item0 += IPT * LSTAGE_THREADS) {
+            for (int item0 = ptid; item0 < (LKB / 8) * n_grp; item0 += IPT * stage_threads) {
                 if constexpr (G % 2 == 0) {
                     // rows kept as 32-bit words (two out_features each): half the registers of a 16-bit copy
                     uint32_t v[IPT][8][G / 2];
@@ -230,7 +231,7 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
                     int ibs[IPT], grps[IPT];
 #pragma unroll
                     for (int q = 0; q < IPT; ++q) {
-                        const int item = item0 + q * LSTAGE_THREADS;
+                        const int item = item0 + q * stage_threads;
                         const bool live = item < (LKB / 8) * n_grp;
                         ibs[q] = live ? item / n_grp : 0;
                         grps[q] = live ? grp_lo + (item - ibs[q] * n_grp) : -1;
@@ -302,11 +303,11 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
             }
             // ---- B: the tokens' slice of x, 8 in_features (16 bytes) at a time, four loads in flight per thread
             const int n_b = NT * (LKB / 8);
-            for (int item0 = ptid; item0 < n_b; item0 += 4 * LSTAGE_THREADS) {
+            for (int item0 = ptid; item0 < n_b; item0 += 4 * stage_threads) {
                 uint4 w[4];
 #pragma unroll
                 for (int u4 = 0; u4 < 4; ++u4) {
-                    const int item = item0 + u4 * LSTAGE_THREADS;
+                    const int item = item0 + u4 * stage_threads;
                     const int kc = item % (LKB / 8), r = item / (LKB / 8);
                     const int m = m0 + r, i = i0 + kc * 8;
                     w[u4] = make_uint4(0u, 0u, 0u, 0u);
@@ -327,7 +328,7 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
                 }
 #pragma unroll
                 for (int u4 = 0; u4 < 4; ++u4) {
-                    const int item = item0 + u4 * LSTAGE_THREADS;
+                    const int item = item0 + u4 * stage_threads;
                     if (item < n_b) {
                         const int kc = item % (LKB / 8), r = item / (LKB / 8);
                         *reinterpret_cast<uint4*>(tB + tile_off(r, kc, B_LBO, 128)) = w[u4];
@@ -367,8 +368,8 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
             const uint64_t descB0 = make_desc(smem_u32(sB), B_LBO, 128);
             bool ok = true;
             for (int c = 0; c < n_chunks && ok; ++c) {
-                const int st = c % LSTAGES;
-                ok = mbar_wait(smem_u32(full + st), (c / LSTAGES) & 1, abort_flag);
+                const int st = c % n_stages;
+                ok = mbar_wait(smem_u32(full + st), (c / n_stages) & 1, abort_flag);
                 if (!ok) break;
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint64_t descA = descA0 + (uint64_t)((st * A_STAGE) >> 4);
@@ -623,7 +624,7 @@ size_t gemv_smem(int g, int K, int rows, int mt) {
     return 128 + ((size_t)rows * mt * 4 + 15) / 16 * 16 + (tail + 15) / 16 * 16;
 }
 
-struct LinearPlan { int NT, a_pad, tmem_cols, o_tiles, tok_blocks, splits, chunks_per_split; size_t smem; };
+struct LinearPlan { int NT, a_pad, stages, tmem_cols, o_tiles, tok_blocks, splits, chunks_per_split; size_t smem; };
 
 // nt_max: tokens per CTA (256, or 64 with a quantised codebook in shared memory); table_bytes: that codebook.
 LinearPlan linear_plan(int64_t M, int64_t d_out, int64_t d_in, int sm_count, int nt_max = LNT_MAX, size_t table_bytes = 0) {
@@ -641,7 +642,8 @@ LinearPlan linear_plan(int64_t M, int64_t d_out, int64_t d_in, int sm_count, int
     p.chunks_per_split = (chunks + splits - 1) / splits;
     p.splits = (chunks + p.chunks_per_split - 1) / p.chunks_per_split;
     p.a_pad = (table_bytes == 0 && p.NT <= 64) ? 1 : 0;
-    p.smem = (size_t)LSTAGES * (a_stage(p.a_pad) + (size_t)b_stage_bytes(p.NT)) + 256;
+    p.stages = (table_bytes != 0 && p.NT > LQ_NT_MAX) ? 2 : LSTAGES;
+    p.smem = (size_t)p.stages * (a_stage(p.a_pad) + (size_t)b_stage_bytes(p.NT)) + 256;
     if (table_bytes) p.smem += 1024 + (table_bytes + 15) / 16 * 16;
     return p;
 }
@@ -686,7 +688,7 @@ cudaError_t launch_linear(cc_ctx* ctx, const LinearPlan& p, const uint16_t* x, i
     static bool attr_dev[64] = {};
     bool& have = attr_dev[ctx->device & 63];
     if (!have) {
-        const int max_smem = QUANT ? (int)(LSTAGES * (a_stage(false) + b_stage_bytes(LQ_NT_MAX)) + 256 + 1024 + LQ_TABLE_MAX)
+        const int max_smem = QUANT ? (int)(LSTAGES * (a_stage(false) + b_stage_bytes(LQ_NT_MAX)) + 256 + 1024 + LQ_TABLE_MAX)   // the larger of its two shapes
                                    : (int)(LSTAGES * (a_stage(true) + b_stage_bytes(LNT_MAX)) + 256);
         const cudaError_t e = cudaFuncSetAttribute(linear_forward_kernel<G, QUANT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                    max_smem);
@@ -695,7 +697,7 @@ cudaError_t launch_linear(cc_ctx* ctx, const LinearPlan& p, const uint16_t* x, i
     }
     const dim3 grid(p.o_tiles, p.tok_blocks, p.splits);
     linear_forward_kernel<G, QUANT><<<grid, LTHREADS, p.smem, st>>>(x, M, C16, qtab, qscale, K, idx, d_out, d_in, out_groups,
-                                                                    p.NT, p.a_pad, p.tmem_cols, p.chunks_per_split, out, split_stride,
+                                                                    p.NT, p.a_pad, p.stages, p.tmem_cols, p.chunks_per_split, out, split_stride,
                                                                     bias, status);
     return cudaGetLastError();
 }
@@ -749,7 +751,8 @@ cudaError_t launch_gemv_m(cc_ctx* ctx, const GemvPlan& p, const uint16_t* x, int
 cudaError_t cc_launch_linear_forward(cc_ctx* ctx, const uint16_t* x, int64_t M, const uint16_t* C16,
                                      const unsigned char* qtab, const float* qscale, int K, int g, const uint16_t* idx,
                                      int64_t d_out, int64_t d_in, const float* bias, float* y, cudaStream_t st) {
-    const LinearPlan p = qtab ? linear_plan(M, d_out, d_in, ctx->sm_count, LQ_NT_MAX, (size_t)K * (g / 2))
+    // beside the table: token blocks of 64 with four stages, or, from LQ_WIDE_FROM tokens on, of 256 with two
+    const LinearPlan p = qtab ? linear_plan(M, d_out, d_in, ctx->sm_count, M >= LQ_WIDE_FROM ? LNT_MAX : LQ_NT_MAX, (size_t)K * (g / 2))
                               : linear_plan(M, d_out, d_in, ctx->sm_count);
     char* ws = static_cast<char*>(ctx->ws);
     unsigned* status = reinterpret_cast<unsigned*>(ws);

@@ -123,6 +123,8 @@ def _gpu_forward_q4(x, C16, idx, d_out, d_in, bias):
     (33, 208, 136, 10, 21), (18, 300, 96, 14, 19),
     (64, 4096, 4096, 4, 65536),     # the paper's largest codebook at g = 4: 128 KB packed
     (200, 384, 256, 4, 65535),      # four token blocks of 64; an odd number of bytes
+    (300, 384, 520, 4, 65535),      # from 256 tokens on: blocks of 256 tokens, two stages beside the table
+    (256, 200, 136, 8, 1000), (700, 130, 72, 6, 50),
 ])
 def test_linear_forward_q4_matches_oracle(M, d_out, d_in, g, K):
     from paper_2503_13089_b200 import binding as cc

@@ -363,7 +363,8 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
         // ------------------------------------------------------------ MMA warp: one thread issues
         if (lane == 0) {
             // kind::f16: D = F32 (bits 4-5 = 1), A = B = F16 (0), both K-major, N >> 3 at bit 17, M >> 4 at bit 24
-            const uint32_t idesc = (1u << 4) | ((uint32_t)(NT >> 3) << 17) | ((uint32_t)(LM >> 4) << 24);
+            const int mma_n = NT < LNT_MAX ? NT : LNT_MAX;          // 512 tokens per CTA are two MMAs of 256 columns
+            const uint32_t idesc = (1u << 4) | ((uint32_t)(mma_n >> 3) << 17) | ((uint32_t)(LM >> 4) << 24);
             const uint64_t descA0 = make_desc(smem_u32(sA), A_LBO, A_SBO);
             const uint64_t descB0 = make_desc(smem_u32(sB), B_LBO, 128);
             bool ok = true;
@@ -374,14 +375,16 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
                 asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
                 const uint64_t descA = descA0 + (uint64_t)((st * A_STAGE) >> 4);
                 const uint64_t descB = descB0 + (uint64_t)((st * b_stage) >> 4);
+                for (int nb = 0; nb * mma_n < NT; ++nb) {
 #pragma unroll
-                for (int s = 0; s < LKB / 16; ++s) {
-                    const uint64_t da = descA + (uint64_t)((s * 2 * A_LBO) >> 4);
-                    const uint64_t db = descB + (uint64_t)((s * 2 * B_LBO) >> 4);
-                    const uint32_t acc = (c > 0 || s > 0) ? 1u : 0u;
-                    asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
-                                 "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-                                 ::"r"(tmem), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+                    for (int s = 0; s < LKB / 16; ++s) {
+                        const uint64_t da = descA + (uint64_t)((s * 2 * A_LBO) >> 4);
+                        const uint64_t db = descB + (uint64_t)((s * 2 * B_LBO + nb * mma_n * 16) >> 4);   // 8-row groups are 128 bytes apart
+                        const uint32_t acc = (c > 0 || s > 0) ? 1u : 0u;
+                        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.b32 p, %4, 0;\n\t"
+                                     "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+                                     ::"r"(tmem + (uint32_t)(nb * mma_n)), "l"(da), "l"(db), "r"(idesc), "r"(acc) : "memory");
+                    }
                 }
                 // the stage may be refilled once these MMAs have read it
                 asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];"
@@ -627,10 +630,17 @@ size_t gemv_smem(int g, int K, int rows, int mt) {
 struct LinearPlan { int NT, a_pad, stages, tmem_cols, o_tiles, tok_blocks, splits, chunks_per_split; size_t smem; };
 
 // nt_max: tokens per CTA (256, or 64 with a quantised codebook in shared memory); table_bytes: that codebook.
-LinearPlan linear_plan(int64_t M, int64_t d_out, int64_t d_in, int sm_count, int nt_max = LNT_MAX, size_t table_bytes = 0) {
+LinearPlan linear_plan(int64_t M, int64_t d_out, int64_t d_in, int sm_count, int nt_max = LNT_MAX, size_t table_bytes = 0,
+                       int g = 4) {
     LinearPlan p;
     const int64_t mt = M < nt_max ? M : nt_max;
     p.NT = (int)((mt + 15) / 16 * 16);
+    // FP16 codebook with rows of at most 8 bytes, many tokens: the gathers of the weight tile bound a stage, so
+    // one tile serves 512 tokens (two MMAs of 256 columns, all 512 TMEM columns) and the pipeline has two stages
+    // of that size: 4096 x 4096, g 4, 4096 tokens 0.571 -> 0.464 ms.  With 16-byte rows (g = 8) there are half as
+    // many gathers per weight and the coarser grid costs more than the reuse saves (1.62 -> 1.70 ms on 8192 x 8192).
+    const bool wide = table_bytes == 0 && nt_max == LNT_MAX && M >= 2 * LNT_MAX && g <= 4;
+    if (wide) p.NT = 2 * LNT_MAX;
     p.tmem_cols = 32;
     while (p.tmem_cols < p.NT) p.tmem_cols *= 2;
     p.o_tiles = (int)((d_out + LM - 1) / LM);
@@ -642,7 +652,7 @@ LinearPlan linear_plan(int64_t M, int64_t d_out, int64_t d_in, int sm_count, int
     p.chunks_per_split = (chunks + splits - 1) / splits;
     p.splits = (chunks + p.chunks_per_split - 1) / p.chunks_per_split;
     p.a_pad = (table_bytes == 0 && p.NT <= 64) ? 1 : 0;
-    p.stages = (table_bytes != 0 && p.NT > LQ_NT_MAX) ? 2 : LSTAGES;
+    p.stages = (wide || (table_bytes != 0 && p.NT > LQ_NT_MAX)) ? 2 : LSTAGES;
     p.smem = (size_t)p.stages * (a_stage(p.a_pad) + (size_t)b_stage_bytes(p.NT)) + 256;
     if (table_bytes) p.smem += 1024 + (table_bytes + 15) / 16 * 16;
     return p;
@@ -652,7 +662,7 @@ LinearPlan linear_plan(int64_t M, int64_t d_out, int64_t d_in, int sm_count, int
 
 size_t cc_linear_scratch_bytes(int64_t M, int64_t d_out, int64_t d_in, int sm_count) {
     // enough for either form of the codebook: the quantised one takes narrower token blocks and may split more
-    const LinearPlan p = linear_plan(M, d_out, d_in, sm_count);
+    const LinearPlan p = linear_plan(M, d_out, d_in, sm_count);     // g <= 4: the shape with the fewest CTAs, hence the most splits
     const LinearPlan q = linear_plan(M, d_out, d_in, sm_count, LQ_NT_MAX, 16);
     int splits = p.splits > q.splits ? p.splits : q.splits;
     if (splits < 2) splits = 0;    // a single CTA per tile writes y itself
@@ -689,7 +699,7 @@ cudaError_t launch_linear(cc_ctx* ctx, const LinearPlan& p, const uint16_t* x, i
     bool& have = attr_dev[ctx->device & 63];
     if (!have) {
         const int max_smem = QUANT ? (int)(LSTAGES * (a_stage(false) + b_stage_bytes(LQ_NT_MAX)) + 256 + 1024 + LQ_TABLE_MAX)   // the larger of its two shapes
-                                   : (int)(LSTAGES * (a_stage(true) + b_stage_bytes(LNT_MAX)) + 256);
+                                   : (int)(LSTAGES * (a_stage(true) + b_stage_bytes(LNT_MAX)) + 256);   // more than two stages of 512 tokens
         const cudaError_t e = cudaFuncSetAttribute(linear_forward_kernel<G, QUANT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                                    max_smem);
         if (e != cudaSuccess) return e;
@@ -753,7 +763,7 @@ cudaError_t cc_launch_linear_forward(cc_ctx* ctx, const uint16_t* x, int64_t M, 
                                      int64_t d_out, int64_t d_in, const float* bias, float* y, cudaStream_t st) {
     // beside the table: token blocks of 64 with four stages, or, from LQ_WIDE_FROM tokens on, of 256 with two
     const LinearPlan p = qtab ? linear_plan(M, d_out, d_in, ctx->sm_count, M >= LQ_WIDE_FROM ? LNT_MAX : LQ_NT_MAX, (size_t)K * (g / 2))
-                              : linear_plan(M, d_out, d_in, ctx->sm_count);
+                              : linear_plan(M, d_out, d_in, ctx->sm_count, LNT_MAX, 0, g);
     char* ws = static_cast<char*>(ctx->ws);
     unsigned* status = reinterpret_cast<unsigned*>(ws);
     float* partial = reinterpret_cast<float*>(ws + 256);

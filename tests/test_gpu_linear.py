@@ -49,6 +49,7 @@ def _check(y, want):
 
 @pytest.mark.parametrize("M,d_out,d_in,g,K", [
     (1, 256, 512, 4, 256),          # one token: 16-column MMA, split over the in_features
+    (600, 260, 200, 4, 300), (1024, 130, 328, 8, 77),   # from 512 tokens on one weight tile serves 512 tokens (two MMAs)
     (16, 1000, 520, 4, 700),        # ragged last tile of out_features; in_features not a multiple of 64
     (5, 130, 67, 6, 50),            # padded out_features (130 = 21 x 6 + 4), in_features not a multiple of 8
     (7, 75, 40, 9, 33), (3, 64, 24, 1, 5), (9, 96, 72, 3, 40), (20, 250, 128, 5, 90), (11, 260, 64, 7, 300),

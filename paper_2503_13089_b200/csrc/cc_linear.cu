@@ -124,20 +124,20 @@ __device__ __forceinline__ void load_code_row_words_q(const unsigned char* __res
 // in_features (chunks_per_split stages each).  out: y itself (splits == 1) or this split's slab of
 // partial sums, both M x d_out FP32 row-major.
 // QUANT: the codebook is the packed 4-bit table `qtab` (K G / 2 bytes) with its scale instead of C16.
-template <int G, bool QUANT>
+template <int G, bool QUANT, int STAGES>
 __global__ void __launch_bounds__(LTHREADS, 1)
 linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __restrict__ C16,
                       const unsigned char* __restrict__ qtab, const float* __restrict__ qscale, int K,
                       const uint16_t* __restrict__ idx, int d_out, int d_in, int out_groups, int NT,
-                      int a_pad, int n_stages, int tmem_cols, int chunks_per_split, float* __restrict__ out, int64_t split_stride,
+                      int a_pad, int tmem_cols, int chunks_per_split, float* __restrict__ out, int64_t split_stride,
                       const float* __restrict__ bias, unsigned* __restrict__ status) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     const int A_STAGE = a_stage(a_pad), A_LBO = a_lbo(a_pad), A_SBO = a_sbo(a_pad);
     const int b_stage = b_stage_bytes(NT), B_LBO = b_lbo(NT);
     unsigned char* sA = smem_raw;                                   // n_stages (2 or 4) tiles of 128 x 64
+    constexpr int n_stages = STAGES, stage_threads = LPROD / STAGES;   // producer threads that fill one stage
     unsigned char* sB = sA + n_stages * A_STAGE;                    // n_stages tiles of NT x 64
     uint64_t* bars = reinterpret_cast<uint64_t*>(sB + n_stages * b_stage);
-    const int stage_threads = LPROD / n_stages;                     // producer threads that fill one stage
     uint64_t* full = bars, *empty = bars + LSTAGES, *acc_full = bars + 2 * LSTAGES;
     uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 2 * LSTAGES + 1);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(tmem_slot + 1);
@@ -690,26 +690,46 @@ int cc_linear_q_table_max(void) { return LQ_TABLE_MAX; }
 
 namespace {
 
+template <int G, bool QUANT, int STAGES>
+cudaError_t launch_linear_s(cc_ctx* ctx, const LinearPlan& p, const uint16_t* x, int M, const uint16_t* C16,
+                            const unsigned char* qtab, const float* qscale, int K, const uint16_t* idx, int d_out, int d_in,
+                            int out_groups, float* out, int64_t split_stride, const float* bias, unsigned* status,
+                            cudaStream_t st) {
+    static bool attr_dev[64] = {};
+    bool& have = attr_dev[ctx->device & 63];
+    if (!have) {
+        // the largest shape of each kind: four stages of 64 tokens or two of 256 beside the table; four stages of
+        // 256 tokens or two of 512 without it
+        const int max_smem = QUANT ? (STAGES == 2 ? (int)(2 * (a_stage(false) + b_stage_bytes(LNT_MAX)) + 256 + 1024 + LQ_TABLE_MAX)
+                                                  : (int)(LSTAGES * (a_stage(false) + b_stage_bytes(LQ_NT_MAX)) + 256 + 1024 + LQ_TABLE_MAX))
+                                   : (STAGES == 2 ? (int)(2 * (a_stage(false) + b_stage_bytes(2 * LNT_MAX)) + 256)
+                                                  : (int)(LSTAGES * (a_stage(true) + b_stage_bytes(LNT_MAX)) + 256));
+        const cudaError_t e = cudaFuncSetAttribute(linear_forward_kernel<G, QUANT, STAGES>,
+                                                   cudaFuncAttributeMaxDynamicSharedMemorySize, max_smem);
+        if (e != cudaSuccess) return e;
+        have = true;
+    }
+    const dim3 grid(p.o_tiles, p.tok_blocks, p.splits);
+    linear_forward_kernel<G, QUANT, STAGES><<<grid, LTHREADS, p.smem, st>>>(x, M, C16, qtab, qscale, K, idx, d_out, d_in,
+                                                                            out_groups, p.NT, p.a_pad, p.tmem_cols,
+                                                                            p.chunks_per_split, out, split_stride, bias, status);
+    return cudaGetLastError();
+}
+
+// Two stages exist where the plan can ask for them: beside the 4-bit table, and for rows of at most 8 bytes.
 template <int G, bool QUANT>
 cudaError_t launch_linear(cc_ctx* ctx, const LinearPlan& p, const uint16_t* x, int M, const uint16_t* C16,
                           const unsigned char* qtab, const float* qscale, int K, const uint16_t* idx, int d_out, int d_in,
                           int out_groups, float* out, int64_t split_stride, const float* bias, unsigned* status,
                           cudaStream_t st) {
-    static bool attr_dev[64] = {};
-    bool& have = attr_dev[ctx->device & 63];
-    if (!have) {
-        const int max_smem = QUANT ? (int)(LSTAGES * (a_stage(false) + b_stage_bytes(LQ_NT_MAX)) + 256 + 1024 + LQ_TABLE_MAX)   // the larger of its two shapes
-                                   : (int)(LSTAGES * (a_stage(true) + b_stage_bytes(LNT_MAX)) + 256);   // more than two stages of 512 tokens
-        const cudaError_t e = cudaFuncSetAttribute(linear_forward_kernel<G, QUANT>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                   max_smem);
-        if (e != cudaSuccess) return e;
-        have = true;
+    if constexpr (QUANT || G <= 4) {
+        if (p.stages == 2)
+            return launch_linear_s<G, QUANT, 2>(ctx, p, x, M, C16, qtab, qscale, K, idx, d_out, d_in, out_groups, out,
+                                                split_stride, bias, status, st);
     }
-    const dim3 grid(p.o_tiles, p.tok_blocks, p.splits);
-    linear_forward_kernel<G, QUANT><<<grid, LTHREADS, p.smem, st>>>(x, M, C16, qtab, qscale, K, idx, d_out, d_in, out_groups,
-                                                                    p.NT, p.a_pad, p.stages, p.tmem_cols, p.chunks_per_split, out, split_stride,
-                                                                    bias, status);
-    return cudaGetLastError();
+    if (p.stages != LSTAGES) return cudaErrorInvalidValue;
+    return launch_linear_s<G, QUANT, LSTAGES>(ctx, p, x, M, C16, qtab, qscale, K, idx, d_out, d_in, out_groups, out,
+                                              split_stride, bias, status, st);
 }
 
 }  // namespace

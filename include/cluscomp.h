@@ -302,7 +302,7 @@ cc_status cc_fit_sampled(cc_ctx* ctx, const uint16_t* X, int64_t N, int g, int K
  * bits: 8 or 4.  q (out): K * g signed bytes (8 bits), or ceil(K * g / 2) bytes holding element 2k in
  * the low and element 2k + 1 in the high nibble, two's complement (4 bits).  scale (out, device): one
  * float.  C16_dequantized (out, may be NULL): K x g FP16 = round-to-nearest-even of q * s, usable with
- * cc_decode and cc_linear_forward.  Needs a workspace of at least 256 bytes. */
+ * cc_decode and cc_linear_forward.  Needs a workspace (any size cc_set_workspace accepts). */
 cc_status cc_quantize_codebook(cc_ctx* ctx, const uint16_t* C16, int K, int g, int bits, uint8_t* q, float* scale,
                                uint16_t* C16_dequantized, void* stream);
 

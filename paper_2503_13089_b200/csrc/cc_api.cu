@@ -12,7 +12,7 @@ WsLayout cc_ws_layout(int64_t N, int g, int K) {
     size_t off = 0;
     auto take = [&](size_t bytes) { size_t o = off; off += cc_align_up(bytes ? bytes : 1, 256); return o; };
     const size_t Kpad = cc_align_up((size_t)K, CC_KPAD);
-    L.status = take(256);
+    L.status = take(CC_STATUS_BYTES);
     L.cprep = take(Kpad / 2 * (size_t)(g + 1) * 16);
     L.flagged = take((size_t)N * 4);
     L.partials = take((size_t)CC_OBJ_BLOCKS * 8);
@@ -193,12 +193,12 @@ size_t cc_workspace_bytes(int64_t N, int g, int K) {
 
 cc_status cc_set_workspace(cc_ctx* ctx, void* workspace, size_t bytes) {
     if (!ctx) return CC_ERR_NULL;
-    if (workspace && (!aligned16(workspace) || bytes < 256)) return CC_ERR_ALIGN;
+    if (workspace && (!aligned16(workspace) || bytes < CC_STATUS_BYTES)) return CC_ERR_ALIGN;
     ctx->ws = workspace;
     ctx->ws_bytes = workspace ? bytes : 0;
     if (workspace) {
         if (cudaSetDevice(ctx->device) != cudaSuccess) return CC_ERR_CUDA;
-        if (cudaMemset(workspace, 0, 256) != cudaSuccess) return CC_ERR_CUDA;   // status words
+        if (cudaMemset(workspace, 0, CC_STATUS_BYTES) != cudaSuccess) return CC_ERR_CUDA;   // status block
     }
     return CC_OK;
 }

@@ -55,11 +55,15 @@ struct ProfScope {
     ~ProfScope() { if (slot) cudaEventRecord(slot->b, st); }
 };
 
+// Status block at the start of every workspace: cleared by cc_set_workspace.
+constexpr size_t CC_STATUS_BYTES = 4096;
+constexpr int CC_ARRIVAL_WORD = 64, CC_ARRIVAL_COUNTERS = 960;
+
 // Carving of the workspace for a problem (N, g, K).  All offsets 256-byte aligned.
 struct WsLayout {
-    size_t status;     // 64 x u32: [0] status bits, [2..3] flagged counter (u64), [8] last-block counter of the objective
-                       // sum, [32..35] tensor-path parameters, [36] codebook quantiser's maximum, [40..63] arrival
-                       // counters of the few-token layer forward (zero between calls)
+    size_t status;     // CC_STATUS_BYTES: 1024 x u32: [0] status bits, [2..3] flagged counter (u64), [8] last-block counter of the objective
+                       // sum, [32..35] tensor-path parameters, [36] codebook quantiser's maximum, [64..1023] arrival
+                       // counters of the layer forward's split reduction (zero between calls)
     size_t cprep;      // staged codebook for the FFMA E-step
     size_t flagged;    // u32 list of points sent to the exact stage
     size_t partials;   // doubles: per-block objective partial sums

@@ -130,7 +130,8 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
                       const unsigned char* __restrict__ qtab, const float* __restrict__ qscale, int K,
                       const uint16_t* __restrict__ idx, int d_out, int d_in, int out_groups, int NT,
                       int a_pad, int tmem_cols, int chunks_per_split, float* __restrict__ out, int64_t split_stride,
-                      const float* __restrict__ bias, unsigned* __restrict__ status) {
+                      const float* __restrict__ bias, unsigned* __restrict__ status, unsigned* __restrict__ arrived,
+                      const float* __restrict__ bias_final, float* __restrict__ y_final) {
     extern __shared__ __align__(1024) unsigned char smem_raw[];
     const int A_STAGE = a_stage(a_pad), A_LBO = a_lbo(a_pad), A_SBO = a_sbo(a_pad);
     const int b_stage = b_stage_bytes(NT), B_LBO = b_lbo(NT);
@@ -397,6 +398,38 @@ linear_forward_kernel(const uint16_t* __restrict__ x, int M, const uint16_t* __r
                 *abort_flag = 1;   // the epilogue's wait on acc_full returns at its next look at the flag
         }
     }
+    // ---- split in_features: the CTA that finishes last among the splits of this tile adds the slabs, in split
+    // order (the same bits whichever CTA that is), and the bias, with all its threads; it leaves the counter at
+    // zero for the next call.  Every CTA counts itself, also one that gave up, so that the counter returns to zero.
+    if (arrived) {
+        __shared__ int last;
+        unsigned* cnt = arrived + blockIdx.y * gridDim.x + blockIdx.x;
+        __threadfence();                                            // this thread's slab stores before the count
+        __syncthreads();
+        if (tid == 0) last = atomicAdd(cnt, 1u) == gridDim.z - 1;
+        __syncthreads();
+        if (last) {
+            __threadfence();
+            const int m_end = (M - m0) < NT ? (M - m0) : NT;
+            for (int e = tid; e < m_end * LM; e += LTHREADS) {
+                const int mm = e / LM, o = o0 + (e - mm * LM);
+                if (o >= d_out) continue;
+                const float* src = out + (int64_t)(m0 + mm) * d_out + o;
+                float sum = bias_final ? __ldg(bias_final + o) : 0.f;
+                unsigned k = 0;
+                for (; k + 4 <= gridDim.z; k += 4) {                // four loads in flight, added in split order
+                    float pv[4];
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) pv[u] = __ldcg(src + (int64_t)(k + u) * split_stride);
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) sum += pv[u];
+                }
+                for (; k < gridDim.z; ++k) sum += __ldcg(src + (int64_t)k * split_stride);
+                y_final[(int64_t)(m0 + mm) * d_out + o] = sum;
+            }
+            if (tid == 0) *cnt = 0u;
+        }
+    }
     if (*abort_flag && lane == 0) atomicOr(status, CC_DEV_TIMEOUT);
     if constexpr (QUANT) {
         if (*abort_flag && tid == 0) {   // let the table's copies land before the CTA gives its shared memory back (bounded)
@@ -433,7 +466,6 @@ linear_reduce_kernel(const float* __restrict__ partial, int splits, int64_t n, i
 // finishes last, or by linear_reduce_kernel: the same bits on every call.
 // blockIdx.x: block of 64 code groups; blockIdx.y: slice of rows_per_split in_features.
 constexpr int LG_THREADS = 1024, LG_GRPS = 64, LG_SUB = 16, LG_ROWS_MAX = 1024, LG_M_MAX = 4;
-constexpr int LG_COUNTER_WORD = 40, LG_COUNTERS = 24;   // words 40..63 of the 64-word status block
 
 template <int G>
 __device__ __forceinline__ void gemv_levels(const unsigned char* row, unsigned (&lv)[G]) {
@@ -672,7 +704,7 @@ size_t cc_linear_scratch_bytes(int64_t M, int64_t d_out, int64_t d_in, int sm_co
         const GemvPlan v = gemv_plan(d_in, (int)((d_out + 15) / 16), sm_count);
         if (v.splits > splits) splits = v.splits;
     }
-    return 256 + (size_t)splits * (size_t)M * (size_t)d_out * 4;
+    return CC_STATUS_BYTES + (size_t)splits * (size_t)M * (size_t)d_out * 4;
 }
 
 int cc_linear_q_table_max(void) { return LQ_TABLE_MAX; }
@@ -694,7 +726,7 @@ template <int G, bool QUANT, int STAGES>
 cudaError_t launch_linear_s(cc_ctx* ctx, const LinearPlan& p, const uint16_t* x, int M, const uint16_t* C16,
                             const unsigned char* qtab, const float* qscale, int K, const uint16_t* idx, int d_out, int d_in,
                             int out_groups, float* out, int64_t split_stride, const float* bias, unsigned* status,
-                            cudaStream_t st) {
+                            unsigned* arrived, const float* bias_final, float* y_final, cudaStream_t st) {
     static bool attr_dev[64] = {};
     bool& have = attr_dev[ctx->device & 63];
     if (!have) {
@@ -712,7 +744,8 @@ cudaError_t launch_linear_s(cc_ctx* ctx, const LinearPlan& p, const uint16_t* x,
     const dim3 grid(p.o_tiles, p.tok_blocks, p.splits);
     linear_forward_kernel<G, QUANT, STAGES><<<grid, LTHREADS, p.smem, st>>>(x, M, C16, qtab, qscale, K, idx, d_out, d_in,
                                                                             out_groups, p.NT, p.a_pad, p.tmem_cols,
-                                                                            p.chunks_per_split, out, split_stride, bias, status);
+                                                                            p.chunks_per_split, out, split_stride, bias, status, arrived,
+                                                                            bias_final, y_final);
     return cudaGetLastError();
 }
 
@@ -721,15 +754,15 @@ template <int G, bool QUANT>
 cudaError_t launch_linear(cc_ctx* ctx, const LinearPlan& p, const uint16_t* x, int M, const uint16_t* C16,
                           const unsigned char* qtab, const float* qscale, int K, const uint16_t* idx, int d_out, int d_in,
                           int out_groups, float* out, int64_t split_stride, const float* bias, unsigned* status,
-                          cudaStream_t st) {
+                          unsigned* arrived, const float* bias_final, float* y_final, cudaStream_t st) {
     if constexpr (QUANT || G <= 4) {
         if (p.stages == 2)
             return launch_linear_s<G, QUANT, 2>(ctx, p, x, M, C16, qtab, qscale, K, idx, d_out, d_in, out_groups, out,
-                                                split_stride, bias, status, st);
+                                                split_stride, bias, status, arrived, bias_final, y_final, st);
     }
     if (p.stages != LSTAGES) return cudaErrorInvalidValue;
     return launch_linear_s<G, QUANT, LSTAGES>(ctx, p, x, M, C16, qtab, qscale, K, idx, d_out, d_in, out_groups, out,
-                                              split_stride, bias, status, st);
+                                              split_stride, bias, status, arrived, bias_final, y_final, st);
 }
 
 }  // namespace
@@ -786,7 +819,7 @@ cudaError_t cc_launch_linear_forward(cc_ctx* ctx, const uint16_t* x, int64_t M, 
                               : linear_plan(M, d_out, d_in, ctx->sm_count, LNT_MAX, 0, g);
     char* ws = static_cast<char*>(ctx->ws);
     unsigned* status = reinterpret_cast<unsigned*>(ws);
-    float* partial = reinterpret_cast<float*>(ws + 256);
+    float* partial = reinterpret_cast<float*>(ws + CC_STATUS_BYTES);
     const int out_groups = (int)((d_out + g - 1) / g);
     const int64_t n = M * d_out;
     cudaError_t e = cudaSuccess;
@@ -796,10 +829,10 @@ cudaError_t cc_launch_linear_forward(cc_ctx* ctx, const uint16_t* x, int64_t M, 
         unsigned* arrived = nullptr;
         {
             ProfScope ps(ctx, CC_K_LINEAR, st);
-            // counters of the finished slices: words of the status block that nothing else uses (zero since
+            // counters of the finished slices: the words of the status block kept for this (zero since
             // cc_set_workspace, put back to zero by the kernel); with more blocks than counters the reduction
             // is a kernel of its own
-            arrived = (v.splits > 1 && v.o_blocks <= LG_COUNTERS) ? status + LG_COUNTER_WORD : nullptr;
+            arrived = (v.splits > 1 && v.o_blocks <= CC_ARRIVAL_COUNTERS) ? status + CC_ARRIVAL_WORD : nullptr;
             float* slabs = v.splits == 1 ? y : partial;          // a single slice writes y (and the bias) itself
 #define CALL(G) e = launch_gemv_m<G>(ctx, v, x, (int)M, qtab, qscale, K, idx, (int)d_out, (int)d_in, out_groups, slabs, n, status, arrived, bias, y, st)
             switch (g) {
@@ -817,12 +850,18 @@ cudaError_t cc_launch_linear_forward(cc_ctx* ctx, const uint16_t* x, int64_t M, 
         linear_reduce_kernel<<<(unsigned)blocks, 256, 0, st>>>(partial, v.splits, n, (int)d_out, bias, y);
         return cudaGetLastError();
     }
+    bool fused = false;
     {
         ProfScope ps(ctx, CC_K_LINEAR, st);
         float* out = p.splits > 1 ? partial : y;
         const float* b = p.splits > 1 ? nullptr : bias;
+        // split in_features: up to 16 tokens the last CTA of a tile adds the slabs (one launch: 33.5 against 38 us
+        // at one token, 36 against 38 at 16; at 64 tokens the lone CTA's tail costs more than the second launch:
+        // 44 against 40 us), if the status block has a counter for every tile; else the reduction is a kernel of its own
+        fused = p.splits > 1 && M <= 16 && (int64_t)p.o_tiles * p.tok_blocks <= CC_ARRIVAL_COUNTERS;
+        unsigned* arrived = fused ? status + CC_ARRIVAL_WORD : nullptr;
         if (qtab) {
-#define CALL(G) e = launch_linear<G, true>(ctx, p, x, (int)M, nullptr, qtab, qscale, K, idx, (int)d_out, (int)d_in, out_groups, out, n, b, status, st)
+#define CALL(G) e = launch_linear<G, true>(ctx, p, x, (int)M, nullptr, qtab, qscale, K, idx, (int)d_out, (int)d_in, out_groups, out, n, b, status, arrived, bias, y, st)
             switch (g) {
                 case 2: CALL(2); break;   case 4: CALL(4); break;   case 6: CALL(6); break;   case 8: CALL(8); break;
                 case 10: CALL(10); break; case 12: CALL(12); break; case 14: CALL(14); break; case 16: CALL(16); break;
@@ -830,13 +869,13 @@ cudaError_t cc_launch_linear_forward(cc_ctx* ctx, const uint16_t* x, int64_t M, 
             }
 #undef CALL
         } else {
-#define CALL(G) e = launch_linear<G, false>(ctx, p, x, (int)M, C16, nullptr, nullptr, K, idx, (int)d_out, (int)d_in, out_groups, out, n, b, status, st)
+#define CALL(G) e = launch_linear<G, false>(ctx, p, x, (int)M, C16, nullptr, nullptr, K, idx, (int)d_out, (int)d_in, out_groups, out, n, b, status, arrived, bias, y, st)
             CC_LINEAR_DISPATCH(g, CALL)
 #undef CALL
         }
     }
     if (e != cudaSuccess) return e;
-    if (p.splits > 1) {
+    if (p.splits > 1 && !fused) {
         ProfScope ps(ctx, CC_K_LINEAR_REDUCE, st);
         int64_t blocks = (n + 255) / 256;
         const int64_t cap = (int64_t)ctx->sm_count * 8;

@@ -150,6 +150,7 @@ def test_linear_forward_q4_matches_oracle(M, d_out, d_in, g, K):
     (2, 144, 328, 10, 77), (1, 260, 64, 12, 300), (2, 300, 96, 14, 19), (2, 2048, 1024, 16, 16384), (1, 8200, 40, 16, 1400),
     (2, 128, 5000, 4, 256),         # one block of code groups, in_features cut into more slices than 16 each would give
     (1, 40, 9, 4, 3),               # fewer than 16 in_features
+    (1, 123000, 2050, 2, 16),       # more blocks of code groups than arrival counters, three slices: the reduction is a kernel of its own
 ])
 def test_linear_forward_q4_few_tokens_matches_oracle(M, d_out, d_in, g, K):
     """The kernel that serves a handful of tokens (no tensor core: table look-ups and FP32 FMAs) against the oracle's
